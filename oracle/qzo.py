@@ -1,0 +1,99 @@
+"""One QZO step (oracle): Algorithm 1, Eq. 5 (Q-SPSA) and Eq. 6 (DDC).
+
+Two forms are given.  `step_literal` walks Algorithm 1 as printed: perturb the
+scales in place by +eps z, forward, by -2 eps z, forward, by +eps z (restore),
+then d, d' and the seeded update with max(., 0).  `step_functional` evaluates
+the same quantities from the untouched scales, Delta' = Delta + sign*eps*z,
+which is what the library does.  In exact arithmetic they agree; the tests
+require agreement to fp64 rounding.
+
+Storage rounding of the updated scale (bf16, ties to even) is a reading: the
+paper does not fix the dtype of Delta.  `lr * d'` is formed once in fp32 and
+the update s - (lr d') z is evaluated in fp32 before rounding, the precision
+the library uses, so that the rounding decision is taken alike on both sides.
+"""
+import numpy as np
+from . import philox
+from .int4 import bf16_round
+from .model import forward_loss, scale_index_bases, LINEAR_ORDER
+
+
+def ddc_clip(d, C):
+    """Eq. 6: d' = C if d > C; d if -C <= d <= C; -C if d < -C  (C >= 0)."""
+    assert C >= 0
+    if d > C:
+        return float(C)
+    if d < -C:
+        return float(-C)
+    return float(d)
+
+
+def directional_derivative(loss_plus, loss_minus, eps):
+    """d = (l+ - l-) / (2 eps), Algorithm 1."""
+    return (loss_plus - loss_minus) / (2.0 * eps)
+
+
+def update_scales_flat(s, seed, index_base, lr, d_clipped):
+    """s_i <- bf16(max(s_i - (lr d') z_i, 0)), fp32 arithmetic (Algorithm 1, last loop)."""
+    s = np.asarray(s, dtype=np.float32)
+    z = philox.normal_range(seed, index_base, s.size).reshape(s.shape)
+    coef = np.float32(np.float32(lr) * np.float32(d_clipped))
+    prod = (coef * z).astype(np.float32)
+    new = np.maximum((s - prod).astype(np.float32), np.float32(0.0))
+    return bf16_round(new)
+
+
+def update_model_scales(model, seed, lr, d_clipped):
+    """Apply the seeded update to every int4 linear of the model, in place."""
+    cfg = model["cfg"]
+    bases, _ = scale_index_bases(cfg)
+    for li, layer in enumerate(model["layers"]):
+        for name in LINEAR_ORDER[cfg["arch"]]:
+            p = layer["lin"][name]
+            p["s"] = update_scales_flat(p["s"], seed, bases[li][name], lr, d_clipped)
+
+
+def step_functional(model, tokens, labels, seed, eps, lr, C, update=True):
+    """One step from the untouched scales; returns (l+, l-, d, d')."""
+    lp = forward_loss(model, tokens, labels, seed, +1, eps)
+    lm = forward_loss(model, tokens, labels, seed, -1, eps)
+    d = directional_derivative(lp, lm, eps)
+    dc = ddc_clip(d, C)
+    if update:
+        update_model_scales(model, seed, lr, dc)
+    return lp, lm, d, dc
+
+
+def _perturb_in_place(model, scale, seed):
+    """PERTURB_SCALES(Delta, scale, s): Delta_i += scale * z_i, fp64, no clamp."""
+    cfg = model["cfg"]
+    bases, _ = scale_index_bases(cfg)
+    for li, layer in enumerate(model["layers"]):
+        for name in LINEAR_ORDER[cfg["arch"]]:
+            p = layer["lin"][name]
+            s = np.asarray(p["s"], dtype=np.float64)
+            z = philox.normal_range(seed, bases[li][name], s.size).astype(np.float64)
+            p["s"] = s + scale * z.reshape(s.shape)
+
+
+def step_literal(model, tokens, labels, seed, eps, lr, C):
+    """Algorithm 1 as printed, scales held in fp64 and mutated in place.
+
+    Returns (l+, l-, d, d'); the model's scales end as fp64
+    max(Delta_i - lr d' z_i, 0) without storage rounding.
+    """
+    _perturb_in_place(model, +eps, seed)
+    lp = forward_loss(model, tokens, labels, seed, 0, eps)
+    _perturb_in_place(model, -2.0 * eps, seed)
+    lm = forward_loss(model, tokens, labels, seed, 0, eps)
+    _perturb_in_place(model, +eps, seed)
+    d = directional_derivative(lp, lm, eps)
+    dc = ddc_clip(d, C)
+    cfg = model["cfg"]
+    bases, _ = scale_index_bases(cfg)
+    for li, layer in enumerate(model["layers"]):
+        for name in LINEAR_ORDER[cfg["arch"]]:
+            p = layer["lin"][name]
+            z = philox.normal_range(seed, bases[li][name], p["s"].size).astype(np.float64)
+            p["s"] = np.maximum(p["s"] - lr * dc * z.reshape(p["s"].shape), 0.0)
+    return lp, lm, d, dc

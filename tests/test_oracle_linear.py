@@ -1,0 +1,57 @@
+"""Pins for oracle/linear.py: brute force, the unperturbed special case, linearity in eps."""
+import numpy as np
+
+from oracle import int4, linear, philox
+
+
+def _case(M=5, K=272, N=12, seed=0):
+    rng = np.random.default_rng(seed)
+    x = rng.standard_normal((M, K))
+    q = rng.integers(-8, 8, size=(K, N)).astype(np.int8)
+    s = int4.bf16_round(rng.uniform(0.005, 0.02, size=(int4.num_groups(K), N)).astype(np.float32))
+    return x, q, s
+
+
+def test_brute_force_tiny():
+    x, q, s = _case(M=3, K=136, N=4)
+    seed, base, eps = 77, 40, 1e-3
+    y = linear.perturbed_linear(x, q, s, seed, base, -1, eps)
+    G, N = s.shape
+    for t in range(3):
+        for n in range(N):
+            acc = 0.0
+            for k in range(136):
+                g = k // 128
+                z = float(philox.normal_from_index(seed, np.array([base + g * N + n]))[0])
+                acc += x[t, k] * (float(s[g, n]) - eps * z) * int(q[k, n])
+            assert abs(acc - y[t, n]) <= 1e-12 * max(1.0, abs(acc))
+
+
+def test_sign_zero_is_textbook_dequant_gemm():
+    x, q, s = _case()
+    y0 = linear.perturbed_linear(x, q, s, 1, 0, 0, 1e-3)
+    np.testing.assert_allclose(y0, x @ int4.dequantize(q, s), rtol=1e-13, atol=1e-13)
+    b = np.linspace(-1, 1, q.shape[1])
+    yb = linear.perturbed_linear(x, q, s, 1, 0, 0, 1e-3, bias=b)
+    np.testing.assert_allclose(yb - y0, np.broadcast_to(b, y0.shape), atol=1e-12)
+
+
+def test_linearity_in_the_perturbation():
+    x, q, s = _case(seed=2)
+    seed, base, eps = 5, 8, 1e-3
+    yp = linear.perturbed_linear(x, q, s, seed, base, +1, eps)
+    ym = linear.perturbed_linear(x, q, s, seed, base, -1, eps)
+    y0 = linear.perturbed_linear(x, q, s, seed, base, 0, eps)
+    np.testing.assert_allclose(yp + ym, 2 * y0, rtol=1e-12, atol=1e-12)
+    z = philox.normal_range(seed, base, s.size).astype(np.float64).reshape(s.shape)
+    zq = z[np.arange(q.shape[0]) // 128] * q
+    np.testing.assert_allclose(yp - ym, 2 * eps * (x @ zq), rtol=1e-9, atol=1e-12)
+    # a different index base draws different noise
+    yp2 = linear.perturbed_linear(x, q, s, seed, base + 8, +1, eps)
+    assert np.abs(yp2 - yp).max() > 0
+
+
+def test_no_clamp_on_perturbed_scales():
+    s = np.full((1, 8), 1e-6, dtype=np.float32)
+    sp = linear.perturbed_scales(s, 3, 0, +1, 1e-3)
+    assert (sp < 0).any()          # Algorithm 1's PERTURB_SCALES has no max(., 0)
