@@ -1,0 +1,203 @@
+/*
+ * qzo.h - C ABI of the QZO hot path on NVIDIA B200 (sm_100a).
+ *
+ * QZO (Quantized Zeroth-order Optimization) fine-tunes a weight-only int4 LLM by
+ * perturbing only its quantisation scales.  One optimisation step (Algorithm 1) is
+ *   l+ = L((Delta + eps z) (.) theta_bar; B)          first forward
+ *   l- = L((Delta - eps z) (.) theta_bar; B)          second forward
+ *   d  = (l+ - l-) / (2 eps),  d' = clip(d, -C, C)    Eq. 5, Eq. 6
+ *   Delta_i <- max(Delta_i - eta d' z_i, 0)           seeded update
+ * with z ~ N(0, I) regenerated from a seed and never stored (Sec. 3.1).
+ *
+ * Conventions
+ *  - Every pointer named d_* is a DEVICE pointer owned by the caller; h_* is a HOST
+ *    pointer.  The library allocates no device memory: model state lives in the
+ *    caller's tensors and in one caller-provided workspace.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *    Calls are asynchronous on that stream unless stated otherwise.
+ *  - Every function returns QZO_OK (0) or a negative qzo_status.  No exceptions cross
+ *    the boundary.  A model handle must not be used from two threads at once.
+ *  - Only compute-capability 10.x devices are supported; there is no CPU or other
+ *    backend (QZO_ERR_UNSUPPORTED_DEVICE).
+ *
+ * Interchange layouts
+ *  - int4 weights, logical q[k][n] in [-8, 7] for Y[t][n] = sum_k X[t][k] W[k][n]:
+ *    uint32 [K/8][N] row-major, nibble j (bits 4j..4j+3) of word [kw][n] holds
+ *    u = q[8 kw + j][n] + 8.  K must be a multiple of 8, N a multiple of 8.
+ *  - scales: bf16 [G][N] row-major, G = ceil(K / 128); group g covers rows
+ *    128 g .. 128 g + 127 (Eq. 3, Eq. 4 with the group of 128 the paper uses).
+ *  - logical scale index of scale [g][n] of a linear: index_base + g N + n.  It selects
+ *    the Gaussian z_i = z(seed, i) (Philox4x32-10, see qzo_normals) and is independent of
+ *    any tiling.  index_base must be a multiple of 4.
+ *  - kernel layout of the int4 weights: produced by qzo_repack_int4; opaque.
+ */
+#ifndef QZO_H_
+#define QZO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  QZO_OK = 0,
+  QZO_ERR_BAD_ARG = -1,            /* null pointer, bad size, sign not in {-1,0,1}, eps <= 0, clip < 0 ... */
+  QZO_ERR_UNSUPPORTED_DEVICE = -2, /* current device is not sm_100 */
+  QZO_ERR_WORKSPACE = -3,          /* workspace too small or misaligned (256 bytes) */
+  QZO_ERR_NONFINITE = -4,          /* a loss or g is NaN/Inf; scales were left untouched */
+  QZO_ERR_DEVICE_TIMEOUT = -5,     /* a bounded device-side wait expired (status word) */
+  QZO_ERR_CUDA = -6,               /* a CUDA call failed; see qzo_last_cuda_error */
+  QZO_ERR_MISSING_TENSOR = -7      /* qzo_init_model: a required tensor was not supplied */
+} qzo_status;
+
+enum { QZO_ARCH_LLAMA = 0, QZO_ARCH_OPT = 1 };
+enum { QZO_DTYPE_BF16 = 0, QZO_DTYPE_F32 = 1, QZO_DTYPE_U32 = 2, QZO_DTYPE_I32 = 3 };
+
+/* Human-readable text of a status code (static storage). */
+const char* qzo_strerror(int status);
+/* cudaError_t value of the last failed CUDA call in this process (0 if none). */
+int qzo_last_cuda_error(void);
+
+/* ------------------------------------------------------------------------------------
+ * Building blocks (each is one step of the path; exported for parity tests and sweeps)
+ * ---------------------------------------------------------------------------------- */
+
+/* Philox4x32-10 words of counter blocks block_base .. block_base+n_blocks-1 under key
+ * `seed` (Sec. 3.1: only the seed is stored).  d_words: uint32 [n_blocks][4].
+ * d_uniforms (may be NULL): float [n_blocks][4], U(x) = ((x >> 9) + 0.5) 2^-23. */
+int qzo_philox_words(uint64_t seed, uint64_t block_base, int64_t n_blocks,
+                     uint32_t* d_words, float* d_uniforms, void* stream);
+
+/* z_i for i = index_base .. index_base+count-1 (Algorithm 1: "z ~ N(0,1)" after the
+ * generator is reset with seed s).  d_z: float [count]. */
+int qzo_normals(uint64_t seed, uint64_t index_base, int64_t count, float* d_z, void* stream);
+
+/* Eq. 3 with Delta = absmax / (2^(4-1) - 1) per group of 128 rows and per column:
+ * d_w float [K][N] -> d_qpacked uint32 [K/8][N] (interchange), d_scales bf16 [G][N].
+ * Scale = bf16(absmax/7); q = clamp(rne(w / scale), -8, 7); zero scale gives q = 0. */
+int qzo_quantize_int4(const float* d_w, int K, int N, uint32_t* d_qpacked, void* d_scales_bf16,
+                      void* stream);
+
+/* Eq. 4 storage: interchange uint32 [K/8][N] -> int8 q [K][N] (for bit-exact checks). */
+int qzo_unpack_int4(const uint32_t* d_qpacked, int K, int N, int8_t* d_q, void* stream);
+
+/* Size in bytes of the kernel-layout copy of a K x N int4 weight. */
+int qzo_repacked_bytes(int K, int N, size_t* bytes);
+/* interchange -> kernel layout (done once; theta_bar is fixed for the whole run,
+ * Algorithm 1 "quantized weights").  d_out: `bytes` from qzo_repacked_bytes, 256-aligned. */
+int qzo_repack_int4(const uint32_t* d_qpacked, int K, int N, void* d_out, size_t out_bytes,
+                    void* stream);
+/* kernel layout -> int8 q [K][N]: what the GEMM's prologue sees (bit-exact check). */
+int qzo_unpack_kernel_layout(const void* d_wq, int K, int N, int8_t* d_q, void* stream);
+
+/* Workspace the GEMM needs for a problem (0 if none; split-K partial sums otherwise). */
+int qzo_gemm_workspace_bytes(int M, int K, int N, size_t* bytes);
+
+/* Perturbed W4A16 linear (Eq. 4 inside Eq. 5):
+ *   Y[t][n] = sum_k X[t][k] (s[k/128][n] + sign eps z_i) q[k][n] (+ bias[n]),
+ *   i = scale_index_base + (k/128) N + n; the perturbed scale is formed in fp32 inside the
+ *   de-quantisation prologue; the stored scales are never modified.
+ * d_x bf16 [M][K] row-major; d_wq kernel layout (qzo_repack_int4); d_scales bf16 [G][N];
+ * d_bias float [N] or NULL; d_y bf16 [M][N].  sign in {-1, 0, +1} (0 = unperturbed).
+ * d_workspace: qzo_gemm_workspace_bytes, 256-aligned (may be NULL when that is 0).
+ * d_status: int on the device, set non-zero if a bounded wait expired (may be NULL). */
+int qzo_perturbed_gemm(const void* d_x_bf16, const void* d_wq, const void* d_scales_bf16,
+                       const float* d_bias, void* d_y_bf16, int M, int K, int N,
+                       uint64_t seed, uint64_t scale_index_base, int sign, float eps,
+                       void* d_workspace, size_t workspace_bytes, int* d_status, void* stream);
+
+/* Seeded update of a flat run of scales (Algorithm 1, last loop, with Eq. 6 applied to g):
+ *   s_i <- bf16(max(s_i - (lr clip(g,-C,C)) z_i, 0)), i = index_base .. index_base+count-1.
+ * d_scales bf16 [count], in place.  g must be finite, clip >= 0. */
+int qzo_update_scales_flat(void* d_scales_bf16, int64_t count, uint64_t seed, uint64_t index_base,
+                           float lr, float g, float clip, void* stream);
+
+/* ------------------------------------------------------------------------------------
+ * Model-level entry points
+ * ---------------------------------------------------------------------------------- */
+
+typedef struct qzo_model qzo_model; /* opaque handle (host memory owned by the library) */
+
+typedef struct {
+  int arch;        /* QZO_ARCH_LLAMA: RMSNorm, RoPE, SiLU-gated MLP, no bias;
+                      QZO_ARCH_OPT: LayerNorm, learned positions, ReLU MLP, biases */
+  int n_layers, d_model, n_heads, d_ffn, vocab, max_seq;
+  int group_size;  /* must be 128 */
+  float norm_eps, rope_theta;
+} qzo_model_desc;
+
+typedef struct {
+  const char* name; /* see qzo_init_model */
+  void* dptr;       /* device pointer */
+  int dtype;        /* QZO_DTYPE_* */
+  int64_t shape[2]; /* rows, cols (cols = 1 for vectors) */
+} qzo_tensor;
+
+/* Number of entries of the flat scale buffer (all block linears, layer-major, in the order
+ * q,k,v,o,gate,up,down (Llama) / q,k,v,o,fc1,fc2 (OPT), each base rounded up to a multiple
+ * of 8) and the number of trainable scales (Table 2: block linear weights / 128). */
+int qzo_num_scales(const qzo_model_desc* desc, int64_t* flat_entries, int64_t* trainable);
+/* Where linear `linear` (position in the order above) of layer `layer` sits in the flat buffer. */
+int qzo_scale_layout(const qzo_model_desc* desc, int layer, int linear,
+                     int64_t* index_base, int* G, int* N);
+
+/* Bytes of workspace qzo_init_model needs for batches up to max_tokens = B*S tokens
+ * (kernel-layout weights + activations + fp32 logits + split-K partials). */
+int qzo_workspace_bytes(const qzo_model_desc* desc, int max_tokens, size_t* bytes);
+
+/* Binds a model to caller-owned tensors (Algorithm 1 "Require": scales Delta, integer
+ * weights theta_bar).  Tensors, by name:
+ *   "embed" bf16 [V][d]; "lm_head" bf16 [V][d]; "pos_embed" bf16 [max_seq][d] (OPT);
+ *   "final_norm_w" f32 [d] (+ "final_norm_b", OPT); "scales" bf16 [flat_entries] (trained in place);
+ *   "L<i>.norm1_w", "L<i>.norm2_w" f32 [d] (+ "_b", OPT);
+ *   "L<i>.<lin>.qweight" u32 [K/8][N] interchange layout (copied into the workspace in kernel
+ *   layout during this call; the caller may free it after the stream has drained);
+ *   "L<i>.<lin>.bias" f32 [N] (OPT).
+ * d_workspace: qzo_workspace_bytes, 256-aligned, must outlive the handle. */
+int qzo_init_model(const qzo_model_desc* desc, const qzo_tensor* tensors, int n_tensors,
+                   void* d_workspace, size_t workspace_bytes, int max_tokens, void* stream,
+                   qzo_model** out);
+int qzo_free_model(qzo_model* m);
+
+/* One forward pass, L(Delta' (.) theta_bar; B) with Delta' = Delta + sign eps z(seed)
+ * (Algorithm 1, "1st/2nd forward pass"; sign 0 = unperturbed).  d_tokens, d_labels:
+ * int32 [B][S]; label -100 is ignored; loss = mean next-token cross entropy over kept
+ * positions, written to d_loss (float, device). */
+int qzo_forward_loss(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S,
+                     uint64_t seed, int sign, float eps, float* d_loss);
+
+/* Seeded update of every scale of the model with a host-side g (clipped here, Eq. 6).
+ * Non-finite g: QZO_ERR_NONFINITE and no write. */
+int qzo_update_scales(qzo_model* m, uint64_t seed, float lr, float g, float clip);
+
+/* Whole step of Algorithm 1 on device-resident tokens: two forwards (sign +1, -1), d, d' and
+ * the update, with d formed on the device.  h_out (may be NULL): {l+, l-, d, d'}; when
+ * non-NULL the call synchronises the stream.  If either loss is not finite the scales are
+ * left untouched and (when h_out is given) QZO_ERR_NONFINITE is returned. */
+int qzo_step(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S,
+             uint64_t seed, float eps, float lr, float clip, float* h_out);
+
+/* Same step with HOST token / label buffers (int32 [B][S]); copies them in, runs the step and
+ * reads {l+, l-, d, d'} back.  Synchronises. */
+int qzo_step_host(qzo_model* m, const int32_t* h_tokens, const int32_t* h_labels, int B, int S,
+                  uint64_t seed, float eps, float lr, float clip, float* h_out);
+
+/* Selects the decoder block whose output later forwards keep a copy of (-1 = none). */
+int qzo_debug_set_capture(qzo_model* m, int layer);
+/* Copies an intermediate of the LAST forward into d_out (bf16 [T][d] for which = 0: output of
+ * decoder block `layer`, which must be the block chosen with qzo_debug_set_capture before that
+ * forward; float [T][V] for which = 1: logits, layer ignored). */
+int qzo_debug_layer_output(qzo_model* m, int layer, int which, void* d_out, size_t bytes);
+
+/* Reads the device status word (0 = no bounded wait has expired since init). Synchronises. */
+int qzo_device_status(qzo_model* m, int* h_status);
+
+/* Number of kernels the library launched since the process started (for benchmark accounting). */
+int64_t qzo_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QZO_H_ */

@@ -1,0 +1,31 @@
+// Launchers of the non-GEMM kernels (layers.cu) and of the GEMMs (gemm_w4a16.cu).
+#pragma once
+#include "qzo_common.cuh"
+
+namespace qzo {
+int launch_embedding(const int32_t* tokens, const __nv_bfloat16* embed, const __nv_bfloat16* pos, int T, int S, int d,
+                     int vocab, __nv_bfloat16* x, cudaStream_t st);
+int launch_rmsnorm(const __nv_bfloat16* x, const float* w, float eps, int T, int d, __nv_bfloat16* y, cudaStream_t st);
+int launch_layernorm(const __nv_bfloat16* x, const float* w, const float* b, float eps, int T, int d,
+                     __nv_bfloat16* y, cudaStream_t st);
+int launch_rope_table(float* cs, int max_seq, int dh, float theta, cudaStream_t st);
+int launch_rope(__nv_bfloat16* q, __nv_bfloat16* k, int ldq, int ldk, const float* cs, int T, int S, int H, int dh,
+                cudaStream_t st);
+int launch_attention(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v, int ldq, int ldk, int ldv,
+                     __nv_bfloat16* out, int ldo, int B, int S, int H, int dh, cudaStream_t st);
+int launch_silu_mul(const __nv_bfloat16* gate, const __nv_bfloat16* up, __nv_bfloat16* out, int64_t n, cudaStream_t st);
+int launch_relu(__nv_bfloat16* x, int64_t n, cudaStream_t st);
+int launch_cross_entropy(const float* logits, const int32_t* labels, int T, int V, float* row_loss, float* loss,
+                         cudaStream_t st);
+int launch_ddc(const float* lp, const float* lm, float eps, float lr, float clip, float* out5, cudaStream_t st);
+
+// gemm_w4a16.cu
+int gemm_splits(int M, int K, int N);
+size_t gemm_workspace_bytes(int M, int K, int N);
+int launch_perturbed_gemm(const __nv_bfloat16* d_x, const void* d_wq, const __nv_bfloat16* d_scales,
+                          const float* d_bias, const __nv_bfloat16* d_residual, __nv_bfloat16* d_y, int ldo,
+                          int M, int K, int N, uint64_t seed, uint64_t idx_base, int sign, float eps,
+                          void* d_ws, size_t ws_bytes, int* d_status, cudaStream_t st);
+int launch_bf16_gemm_f32out(const __nv_bfloat16* d_x, const __nv_bfloat16* d_w, float* d_out, int M, int K, int N,
+                            int* d_status, cudaStream_t st);
+}  // namespace qzo

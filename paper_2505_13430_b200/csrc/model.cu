@@ -1,0 +1,526 @@
+// Host orchestration of the model-level entry points: binds caller-owned tensors, lays the
+// workspace out, and issues the launch sequence of one forward pass and of one QZO step
+// (Algorithm 1) on the caller's stream.  No device memory is allocated here.
+#include "qzo_common.cuh"
+#include "launch.cuh"
+#include "layers.cuh"
+
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <string>
+#include <vector>
+
+namespace qzo {
+
+static std::atomic<int> g_last_cuda_error{0};
+static std::atomic<long long> g_launches{0};
+void set_last_cuda_error(cudaError_t e) { g_last_cuda_error.store((int)e); }
+int last_cuda_error() { return g_last_cuda_error.load(); }
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+long long launch_count() { return g_launches.load(); }
+
+int check_device() {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) { set_last_cuda_error(e); return QZO_ERR_UNSUPPORTED_DEVICE; }
+  int major = 0;
+  e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+  if (e != cudaSuccess) { set_last_cuda_error(e); return QZO_ERR_UNSUPPORTED_DEVICE; }
+  return major == 10 ? QZO_OK : QZO_ERR_UNSUPPORTED_DEVICE;
+}
+
+struct LinearShape { const char* name; int K, N; };
+
+static int linear_shapes(const qzo_model_desc& d, LinearShape out[7]) {
+  const int dm = d.d_model, f = d.d_ffn;
+  if (d.arch == QZO_ARCH_LLAMA) {
+    const LinearShape s[7] = {{"q", dm, dm}, {"k", dm, dm}, {"v", dm, dm}, {"o", dm, dm},
+                              {"gate", dm, f}, {"up", dm, f}, {"down", f, dm}};
+    memcpy(out, s, sizeof(s));
+    return 7;
+  }
+  const LinearShape s[6] = {{"q", dm, dm}, {"k", dm, dm}, {"v", dm, dm}, {"o", dm, dm}, {"fc1", dm, f}, {"fc2", f, dm}};
+  memcpy(out, s, sizeof(s));
+  return 6;
+}
+
+int validate_desc(const qzo_model_desc* d) {
+  if (!d) return QZO_ERR_BAD_ARG;
+  if (d->arch != QZO_ARCH_LLAMA && d->arch != QZO_ARCH_OPT) return QZO_ERR_BAD_ARG;
+  if (d->n_layers <= 0 || d->d_model <= 0 || d->n_heads <= 0 || d->d_ffn <= 0 || d->vocab <= 0 || d->max_seq <= 0)
+    return QZO_ERR_BAD_ARG;
+  if (d->group_size != kGroup) return QZO_ERR_BAD_ARG;
+  if (d->d_model % d->n_heads) return QZO_ERR_BAD_ARG;
+  const int dh = d->d_model / d->n_heads;
+  if (dh != 64 && dh != 128) return QZO_ERR_BAD_ARG;
+  if ((d->d_model % 8) || (d->d_ffn % 8)) return QZO_ERR_BAD_ARG;
+  if (!(d->norm_eps > 0.0f)) return QZO_ERR_BAD_ARG;
+  if (d->arch == QZO_ARCH_LLAMA && !(d->rope_theta > 0.0f)) return QZO_ERR_BAD_ARG;
+  return QZO_OK;
+}
+
+// Index base of (layer, linear) and running total, bases rounded up to a multiple of 8.
+int64_t scale_layout(const qzo_model_desc& d, int layer, int linear, int* G, int* N, int64_t* trainable) {
+  LinearShape ls[7];
+  const int nl = linear_shapes(d, ls);
+  int64_t run = 0, train = 0, found = -1;
+  for (int L = 0; L < d.n_layers; ++L) {
+    for (int i = 0; i < nl; ++i) {
+      run = (run + 7) / 8 * 8;
+      const int g = ceil_div(ls[i].K, kGroup);
+      if (L == layer && i == linear) {
+        found = run;
+        if (G) *G = g;
+        if (N) *N = ls[i].N;
+      }
+      run += (int64_t)g * ls[i].N;
+      train += (int64_t)g * ls[i].N;
+    }
+  }
+  if (trainable) *trainable = train;
+  return (layer < 0) ? run : found;
+}
+
+struct Linear {
+  int K = 0, N = 0;
+  int64_t idx_base = 0;
+  const void* wq = nullptr;     // kernel layout, inside the workspace
+  const float* bias = nullptr;
+};
+struct Layer {
+  const float *norm1_w = nullptr, *norm1_b = nullptr, *norm2_w = nullptr, *norm2_b = nullptr;
+  Linear lin[7];
+};
+
+}  // namespace qzo
+
+struct qzo_model {
+  qzo_model_desc desc;
+  int n_lin = 0;
+  std::vector<qzo::Layer> layers;
+  const __nv_bfloat16 *embed = nullptr, *lm_head = nullptr, *pos_embed = nullptr;
+  const float *final_norm_w = nullptr, *final_norm_b = nullptr;
+  __nv_bfloat16* scales = nullptr;
+  int64_t flat_entries = 0;
+  int max_tokens = 0;
+  cudaStream_t stream = nullptr;
+  // workspace regions
+  __nv_bfloat16 *x = nullptr, *xn = nullptr, *qkv = nullptr, *att = nullptr, *mlp_a = nullptr, *mlp_b = nullptr,
+                *capture = nullptr;
+  float *logits = nullptr, *row_loss = nullptr, *loss2 = nullptr, *out5 = nullptr, *rope_cs = nullptr;
+  int32_t *tok_dev = nullptr, *lab_dev = nullptr;
+  void* gemm_ws = nullptr;
+  size_t gemm_ws_bytes = 0;
+  int* status = nullptr;
+  int capture_layer = -1;
+  int last_T = 0;
+};
+
+namespace qzo {
+
+struct WsPlan {
+  size_t off_weights, off_x, off_xn, off_qkv, off_att, off_a, off_b, off_capture, off_logits, off_rowloss, off_scalars,
+      off_rope, off_tok, off_lab, off_gemm, gemm_bytes, total;
+};
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+int plan_workspace(const qzo_model_desc& d, int T, WsPlan* p) {
+  LinearShape ls[7];
+  const int nl = linear_shapes(d, ls);
+  size_t off = 0;
+  p->off_weights = off;
+  size_t per_layer = 0;
+  for (int i = 0; i < nl; ++i) per_layer += align_up(repacked_bytes(ls[i].K, ls[i].N), 256);
+  off += per_layer * d.n_layers;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  const size_t dm = d.d_model, f = d.d_ffn;
+  p->off_x = take((size_t)T * dm * 2);
+  p->off_xn = take((size_t)T * dm * 2);
+  p->off_qkv = take((size_t)T * 3 * dm * 2);
+  p->off_att = take((size_t)T * dm * 2);
+  p->off_a = take((size_t)T * f * 2);
+  p->off_b = take((size_t)T * f * 2);
+  p->off_capture = take((size_t)T * dm * 2);
+  p->off_logits = take((size_t)T * d.vocab * 4);
+  p->off_rowloss = take((size_t)T * 4);
+  p->off_scalars = take(64 * 4);
+  p->off_rope = take((size_t)d.max_seq * (dm / d.n_heads) * 4);
+  p->off_tok = take((size_t)T * 4);
+  p->off_lab = take((size_t)T * 4);
+  size_t gb = 0;
+  for (int i = 0; i < nl; ++i) gb = std::max(gb, gemm_workspace_bytes(T, ls[i].K, ls[i].N));
+  p->gemm_bytes = gb;
+  p->off_gemm = take(gb);
+  p->total = off;
+  return QZO_OK;
+}
+
+static int norm(const qzo_model* m, const __nv_bfloat16* in, const float* w, const float* b, int T, __nv_bfloat16* out) {
+  if (m->desc.arch == QZO_ARCH_LLAMA) return launch_rmsnorm(in, w, m->desc.norm_eps, T, m->desc.d_model, out, m->stream);
+  return launch_layernorm(in, w, b, m->desc.norm_eps, T, m->desc.d_model, out, m->stream);
+}
+
+static int linear(const qzo_model* m, const Linear& L, const __nv_bfloat16* in, const __nv_bfloat16* residual,
+                  __nv_bfloat16* out, int ldo, int T, uint64_t seed, int sign, float eps) {
+  return launch_perturbed_gemm(in, L.wq, m->scales + L.idx_base, L.bias, residual, out, ldo, T, L.K, L.N, seed,
+                               (uint64_t)L.idx_base, sign, eps, m->gemm_ws, m->gemm_ws_bytes, m->status, m->stream);
+}
+
+int forward_loss(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S, uint64_t seed, int sign,
+                 float eps, float* d_loss) {
+  const qzo_model_desc& d = m->desc;
+  const int T = B * S, dm = d.d_model, H = d.n_heads, dh = dm / H, F = d.d_ffn;
+  cudaStream_t st = m->stream;
+  const bool llama = d.arch == QZO_ARCH_LLAMA;
+  QZO_TRY(launch_embedding(d_tokens, m->embed, llama ? nullptr : m->pos_embed, T, S, dm, d.vocab, m->x, st));
+  for (int li = 0; li < d.n_layers; ++li) {
+    const Layer& L = m->layers[li];
+    QZO_TRY(norm(m, m->x, L.norm1_w, L.norm1_b, T, m->xn));
+    for (int j = 0; j < 3; ++j)
+      QZO_TRY(linear(m, L.lin[j], m->xn, nullptr, m->qkv + (size_t)j * dm, 3 * dm, T, seed, sign, eps));
+    if (llama) QZO_TRY(launch_rope(m->qkv, m->qkv + dm, 3 * dm, 3 * dm, m->rope_cs, T, S, H, dh, st));
+    QZO_TRY(launch_attention(m->qkv, m->qkv + dm, m->qkv + 2 * dm, 3 * dm, 3 * dm, 3 * dm, m->att, dm, B, S, H, dh, st));
+    QZO_TRY(linear(m, L.lin[3], m->att, m->x, m->x, dm, T, seed, sign, eps));
+    QZO_TRY(norm(m, m->x, L.norm2_w, L.norm2_b, T, m->xn));
+    if (llama) {
+      QZO_TRY(linear(m, L.lin[4], m->xn, nullptr, m->mlp_a, F, T, seed, sign, eps));
+      QZO_TRY(linear(m, L.lin[5], m->xn, nullptr, m->mlp_b, F, T, seed, sign, eps));
+      QZO_TRY(launch_silu_mul(m->mlp_a, m->mlp_b, m->mlp_a, (int64_t)T * F, st));
+      QZO_TRY(linear(m, L.lin[6], m->mlp_a, m->x, m->x, dm, T, seed, sign, eps));
+    } else {
+      QZO_TRY(linear(m, L.lin[4], m->xn, nullptr, m->mlp_a, F, T, seed, sign, eps));
+      QZO_TRY(launch_relu(m->mlp_a, (int64_t)T * F, st));
+      QZO_TRY(linear(m, L.lin[5], m->mlp_a, m->x, m->x, dm, T, seed, sign, eps));
+    }
+    if (li == m->capture_layer)
+      QZO_CUDA_TRY(cudaMemcpyAsync(m->capture, m->x, (size_t)T * dm * 2, cudaMemcpyDeviceToDevice, st));
+  }
+  QZO_TRY(norm(m, m->x, m->final_norm_w, m->final_norm_b, T, m->xn));
+  QZO_TRY(launch_bf16_gemm_f32out(m->xn, m->lm_head, m->logits, T, dm, d.vocab, m->status, st));
+  QZO_TRY(launch_cross_entropy(m->logits, d_labels, T, d.vocab, m->row_loss, d_loss, st));
+  m->last_T = T;
+  return QZO_OK;
+}
+
+int check_batch(const qzo_model* m, const void* tok, const void* lab, int B, int S) {
+  if (!m || !tok || !lab || B <= 0 || S <= 0) return QZO_ERR_BAD_ARG;
+  if (S > m->desc.max_seq) return QZO_ERR_BAD_ARG;
+  if ((int64_t)B * S > m->max_tokens) return QZO_ERR_WORKSPACE;
+  return QZO_OK;
+}
+
+int update_all_scales(qzo_model* m, uint64_t seed, float coef_host, const float* coef_dev) {
+  return launch_update_scales(m->scales, m->flat_entries, seed, 0, coef_host, coef_dev, m->stream);
+}
+
+int step_device(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S, uint64_t seed, float eps,
+                float lr, float clip, float* h_out) {
+  QZO_TRY(forward_loss(m, d_tokens, d_labels, B, S, seed, +1, eps, m->loss2));
+  QZO_TRY(forward_loss(m, d_tokens, d_labels, B, S, seed, -1, eps, m->loss2 + 1));
+  QZO_TRY(launch_ddc(m->loss2, m->loss2 + 1, eps, lr, clip, m->out5, m->stream));
+  QZO_TRY(update_all_scales(m, seed, 0.0f, m->out5 + 4));
+  if (h_out) {
+    QZO_CUDA_TRY(cudaMemcpyAsync(h_out, m->out5, 4 * sizeof(float), cudaMemcpyDeviceToHost, m->stream));
+    QZO_CUDA_TRY(cudaStreamSynchronize(m->stream));
+    if (!std::isfinite(h_out[0]) || !std::isfinite(h_out[1])) return QZO_ERR_NONFINITE;
+  }
+  return QZO_OK;
+}
+
+}  // namespace qzo
+
+// =========================================================================================
+// C ABI
+// =========================================================================================
+using namespace qzo;
+
+extern "C" {
+
+const char* qzo_strerror(int status) {
+  switch (status) {
+    case QZO_OK: return "ok";
+    case QZO_ERR_BAD_ARG: return "bad argument";
+    case QZO_ERR_UNSUPPORTED_DEVICE: return "unsupported device (needs compute capability 10.x; no other backend)";
+    case QZO_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case QZO_ERR_NONFINITE: return "non-finite loss or directional derivative; scales untouched";
+    case QZO_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+    case QZO_ERR_CUDA: return "CUDA call failed (see qzo_last_cuda_error)";
+    case QZO_ERR_MISSING_TENSOR: return "a required tensor was not supplied";
+    default: return "unknown status";
+  }
+}
+
+int qzo_last_cuda_error(void) { return qzo::last_cuda_error(); }
+int64_t qzo_launch_count(void) { return (int64_t)qzo::launch_count(); }
+
+int qzo_philox_words(uint64_t seed, uint64_t block_base, int64_t n_blocks, uint32_t* d_words, float* d_uniforms,
+                     void* stream) {
+  if (n_blocks < 0 || (n_blocks > 0 && !d_words)) return QZO_ERR_BAD_ARG;
+  QZO_TRY(check_device());
+  return launch_philox_words(seed, block_base, n_blocks, d_words, d_uniforms, (cudaStream_t)stream);
+}
+
+int qzo_normals(uint64_t seed, uint64_t index_base, int64_t count, float* d_z, void* stream) {
+  if (count < 0 || (count > 0 && !d_z)) return QZO_ERR_BAD_ARG;
+  QZO_TRY(check_device());
+  return launch_normals(seed, index_base, count, d_z, (cudaStream_t)stream);
+}
+
+int qzo_quantize_int4(const float* d_w, int K, int N, uint32_t* d_qpacked, void* d_scales_bf16, void* stream) {
+  if (!d_w || !d_qpacked || !d_scales_bf16 || K <= 0 || N <= 0 || (K % 8)) return QZO_ERR_BAD_ARG;
+  QZO_TRY(check_device());
+  return launch_quantize(d_w, K, N, d_qpacked, (__nv_bfloat16*)d_scales_bf16, (cudaStream_t)stream);
+}
+
+int qzo_unpack_int4(const uint32_t* d_qpacked, int K, int N, int8_t* d_q, void* stream) {
+  if (!d_qpacked || !d_q || K <= 0 || N <= 0 || (K % 8)) return QZO_ERR_BAD_ARG;
+  QZO_TRY(check_device());
+  return launch_unpack(d_qpacked, K, N, d_q, (cudaStream_t)stream);
+}
+
+int qzo_repacked_bytes(int K, int N, size_t* bytes) {
+  if (!bytes || K <= 0 || N <= 0 || (K % 8)) return QZO_ERR_BAD_ARG;
+  *bytes = repacked_bytes(K, N);
+  return QZO_OK;
+}
+
+int qzo_repack_int4(const uint32_t* d_qpacked, int K, int N, void* d_out, size_t out_bytes, void* stream) {
+  if (!d_qpacked || !d_out || K <= 0 || N <= 0 || (K % 8)) return QZO_ERR_BAD_ARG;
+  if (out_bytes < repacked_bytes(K, N) || ((uintptr_t)d_out & 255)) return QZO_ERR_WORKSPACE;
+  QZO_TRY(check_device());
+  return launch_repack(d_qpacked, K, N, d_out, (cudaStream_t)stream);
+}
+
+int qzo_unpack_kernel_layout(const void* d_wq, int K, int N, int8_t* d_q, void* stream) {
+  if (!d_wq || !d_q || K <= 0 || N <= 0 || (K % 8)) return QZO_ERR_BAD_ARG;
+  QZO_TRY(check_device());
+  return launch_unpack_kernel_layout(d_wq, K, N, d_q, (cudaStream_t)stream);
+}
+
+int qzo_gemm_workspace_bytes(int M, int K, int N, size_t* bytes) {
+  if (!bytes || M <= 0 || K <= 0 || N <= 0) return QZO_ERR_BAD_ARG;
+  *bytes = gemm_workspace_bytes(M, K, N);
+  return QZO_OK;
+}
+
+int qzo_perturbed_gemm(const void* d_x_bf16, const void* d_wq, const void* d_scales_bf16, const float* d_bias,
+                       void* d_y_bf16, int M, int K, int N, uint64_t seed, uint64_t scale_index_base, int sign,
+                       float eps, void* d_workspace, size_t workspace_bytes, int* d_status, void* stream) {
+  if (!d_x_bf16 || !d_wq || !d_scales_bf16 || !d_y_bf16) return QZO_ERR_BAD_ARG;
+  if (sign < -1 || sign > 1 || !(eps > 0.0f)) return QZO_ERR_BAD_ARG;
+  if (((uintptr_t)d_x_bf16 & 15) || ((uintptr_t)d_wq & 15) || ((uintptr_t)d_scales_bf16 & 15)) return QZO_ERR_BAD_ARG;
+  if (d_workspace && ((uintptr_t)d_workspace & 255)) return QZO_ERR_WORKSPACE;
+  QZO_TRY(check_device());
+  return launch_perturbed_gemm((const __nv_bfloat16*)d_x_bf16, d_wq, (const __nv_bfloat16*)d_scales_bf16, d_bias,
+                               nullptr, (__nv_bfloat16*)d_y_bf16, N, M, K, N, seed, scale_index_base, sign, eps,
+                               d_workspace, workspace_bytes, d_status, (cudaStream_t)stream);
+}
+
+int qzo_update_scales_flat(void* d_scales_bf16, int64_t count, uint64_t seed, uint64_t index_base, float lr, float g,
+                           float clip, void* stream) {
+  if (!d_scales_bf16 || count < 0 || (index_base % 4) || ((uintptr_t)d_scales_bf16 & 7) || !(clip >= 0.0f))
+    return QZO_ERR_BAD_ARG;
+  if (!std::isfinite(g) || !std::isfinite(lr)) return QZO_ERR_NONFINITE;
+  QZO_TRY(check_device());
+  const float gc = fminf(fmaxf(g, -clip), clip);
+  const float coef = lr * gc;
+  return launch_update_scales((__nv_bfloat16*)d_scales_bf16, count, seed, index_base, coef, nullptr, (cudaStream_t)stream);
+}
+
+int qzo_num_scales(const qzo_model_desc* desc, int64_t* flat_entries, int64_t* trainable) {
+  QZO_TRY(validate_desc(desc));
+  int64_t train = 0;
+  const int64_t flat = scale_layout(*desc, -1, -1, nullptr, nullptr, &train);
+  if (flat_entries) *flat_entries = flat;
+  if (trainable) *trainable = train;
+  return QZO_OK;
+}
+
+int qzo_scale_layout(const qzo_model_desc* desc, int layer, int linear, int64_t* index_base, int* G, int* N) {
+  QZO_TRY(validate_desc(desc));
+  LinearShape ls[7];
+  const int nl = linear_shapes(*desc, ls);
+  if (layer < 0 || layer >= desc->n_layers || linear < 0 || linear >= nl) return QZO_ERR_BAD_ARG;
+  const int64_t b = scale_layout(*desc, layer, linear, G, N, nullptr);
+  if (index_base) *index_base = b;
+  return QZO_OK;
+}
+
+int qzo_workspace_bytes(const qzo_model_desc* desc, int max_tokens, size_t* bytes) {
+  QZO_TRY(validate_desc(desc));
+  if (!bytes || max_tokens <= 0) return QZO_ERR_BAD_ARG;
+  WsPlan p;
+  QZO_TRY(plan_workspace(*desc, max_tokens, &p));
+  *bytes = p.total;
+  return QZO_OK;
+}
+
+int qzo_init_model(const qzo_model_desc* desc, const qzo_tensor* tensors, int n_tensors, void* d_workspace,
+                   size_t workspace_bytes, int max_tokens, void* stream, qzo_model** out) {
+  QZO_TRY(validate_desc(desc));
+  if (!tensors || n_tensors <= 0 || !out || max_tokens <= 0) return QZO_ERR_BAD_ARG;
+  if (!d_workspace || ((uintptr_t)d_workspace & 255)) return QZO_ERR_WORKSPACE;
+  QZO_TRY(check_device());
+  WsPlan p;
+  QZO_TRY(plan_workspace(*desc, max_tokens, &p));
+  if (workspace_bytes < p.total) return QZO_ERR_WORKSPACE;
+
+  std::map<std::string, const qzo_tensor*> by_name;
+  for (int i = 0; i < n_tensors; ++i)
+    if (tensors[i].name && tensors[i].dptr) by_name[tensors[i].name] = &tensors[i];
+  int err = QZO_OK;
+  auto get = [&](const std::string& name, int dtype, int64_t rows, int64_t cols) -> void* {
+    auto it = by_name.find(name);
+    if (it == by_name.end()) { if (err == QZO_OK) err = QZO_ERR_MISSING_TENSOR; return nullptr; }
+    const qzo_tensor* t = it->second;
+    if (t->dtype != dtype || t->shape[0] != rows || t->shape[1] != cols || ((uintptr_t)t->dptr & 15)) {
+      if (err == QZO_OK) err = QZO_ERR_BAD_ARG;
+      return nullptr;
+    }
+    return t->dptr;
+  };
+
+  qzo_model* m = new qzo_model();
+  m->desc = *desc;
+  m->stream = (cudaStream_t)stream;
+  m->max_tokens = max_tokens;
+  const bool opt = desc->arch == QZO_ARCH_OPT;
+  const int dm = desc->d_model;
+  int64_t train = 0;
+  m->flat_entries = scale_layout(*desc, -1, -1, nullptr, nullptr, &train);
+  m->embed = (const __nv_bfloat16*)get("embed", QZO_DTYPE_BF16, desc->vocab, dm);
+  m->lm_head = (const __nv_bfloat16*)get("lm_head", QZO_DTYPE_BF16, desc->vocab, dm);
+  if (opt) m->pos_embed = (const __nv_bfloat16*)get("pos_embed", QZO_DTYPE_BF16, desc->max_seq, dm);
+  m->final_norm_w = (const float*)get("final_norm_w", QZO_DTYPE_F32, dm, 1);
+  if (opt) m->final_norm_b = (const float*)get("final_norm_b", QZO_DTYPE_F32, dm, 1);
+  m->scales = (__nv_bfloat16*)get("scales", QZO_DTYPE_BF16, m->flat_entries, 1);
+
+  uint8_t* ws = (uint8_t*)d_workspace;
+  LinearShape ls[7];
+  m->n_lin = linear_shapes(*desc, ls);
+  m->layers.resize(desc->n_layers);
+  size_t woff = p.off_weights;
+  for (int li = 0; li < desc->n_layers && err == QZO_OK; ++li) {
+    Layer& L = m->layers[li];
+    const std::string pre = "L" + std::to_string(li) + ".";
+    L.norm1_w = (const float*)get(pre + "norm1_w", QZO_DTYPE_F32, dm, 1);
+    L.norm2_w = (const float*)get(pre + "norm2_w", QZO_DTYPE_F32, dm, 1);
+    if (opt) {
+      L.norm1_b = (const float*)get(pre + "norm1_b", QZO_DTYPE_F32, dm, 1);
+      L.norm2_b = (const float*)get(pre + "norm2_b", QZO_DTYPE_F32, dm, 1);
+    }
+    for (int i = 0; i < m->n_lin; ++i) {
+      Linear& lin = L.lin[i];
+      lin.K = ls[i].K; lin.N = ls[i].N;
+      lin.idx_base = scale_layout(*desc, li, i, nullptr, nullptr, nullptr);
+      const uint32_t* qw = (const uint32_t*)get(pre + ls[i].name + ".qweight", QZO_DTYPE_U32, lin.K / 8, lin.N);
+      if (opt) lin.bias = (const float*)get(pre + ls[i].name + ".bias", QZO_DTYPE_F32, lin.N, 1);
+      if (err != QZO_OK) break;
+      lin.wq = ws + woff;
+      int s = launch_repack(qw, lin.K, lin.N, ws + woff, m->stream);
+      if (s != QZO_OK) { err = s; break; }
+      woff += align_up(repacked_bytes(lin.K, lin.N), 256);
+    }
+  }
+  if (err != QZO_OK) { delete m; return err; }
+
+  m->x = (__nv_bfloat16*)(ws + p.off_x);
+  m->xn = (__nv_bfloat16*)(ws + p.off_xn);
+  m->qkv = (__nv_bfloat16*)(ws + p.off_qkv);
+  m->att = (__nv_bfloat16*)(ws + p.off_att);
+  m->mlp_a = (__nv_bfloat16*)(ws + p.off_a);
+  m->mlp_b = (__nv_bfloat16*)(ws + p.off_b);
+  m->capture = (__nv_bfloat16*)(ws + p.off_capture);
+  m->logits = (float*)(ws + p.off_logits);
+  m->row_loss = (float*)(ws + p.off_rowloss);
+  float* scal = (float*)(ws + p.off_scalars);
+  m->loss2 = scal;            // [0], [1]
+  m->out5 = scal + 8;         // [8..12]
+  m->status = (int*)(scal + 32);
+  m->rope_cs = (float*)(ws + p.off_rope);
+  m->tok_dev = (int32_t*)(ws + p.off_tok);
+  m->lab_dev = (int32_t*)(ws + p.off_lab);
+  m->gemm_ws = ws + p.off_gemm;
+  m->gemm_ws_bytes = p.gemm_bytes;
+  cudaError_t ce = cudaMemsetAsync(scal, 0, 64 * 4, m->stream);
+  if (ce != cudaSuccess) { set_last_cuda_error(ce); delete m; return QZO_ERR_CUDA; }
+  if (!opt) {
+    int s = launch_rope_table(m->rope_cs, desc->max_seq, dm / desc->n_heads, desc->rope_theta, m->stream);
+    if (s != QZO_OK) { delete m; return s; }
+  }
+  *out = m;
+  return QZO_OK;
+}
+
+int qzo_free_model(qzo_model* m) {
+  if (!m) return QZO_ERR_BAD_ARG;
+  delete m;
+  return QZO_OK;
+}
+
+int qzo_forward_loss(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S, uint64_t seed,
+                     int sign, float eps, float* d_loss) {
+  QZO_TRY(check_batch(m, d_tokens, d_labels, B, S));
+  if (!d_loss || sign < -1 || sign > 1 || !(eps > 0.0f)) return QZO_ERR_BAD_ARG;
+  return forward_loss(m, d_tokens, d_labels, B, S, seed, sign, eps, d_loss);
+}
+
+int qzo_update_scales(qzo_model* m, uint64_t seed, float lr, float g, float clip) {
+  if (!m || !(clip >= 0.0f)) return QZO_ERR_BAD_ARG;
+  if (!std::isfinite(g) || !std::isfinite(lr)) return QZO_ERR_NONFINITE;
+  const float gc = fminf(fmaxf(g, -clip), clip);
+  return update_all_scales(m, seed, lr * gc, nullptr);
+}
+
+int qzo_step(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S, uint64_t seed, float eps,
+             float lr, float clip, float* h_out) {
+  QZO_TRY(check_batch(m, d_tokens, d_labels, B, S));
+  if (!(eps > 0.0f) || !(clip >= 0.0f) || !std::isfinite(lr)) return QZO_ERR_BAD_ARG;
+  return step_device(m, d_tokens, d_labels, B, S, seed, eps, lr, clip, h_out);
+}
+
+int qzo_step_host(qzo_model* m, const int32_t* h_tokens, const int32_t* h_labels, int B, int S, uint64_t seed,
+                  float eps, float lr, float clip, float* h_out) {
+  QZO_TRY(check_batch(m, h_tokens, h_labels, B, S));
+  if (!(eps > 0.0f) || !(clip >= 0.0f) || !std::isfinite(lr) || !h_out) return QZO_ERR_BAD_ARG;
+  const size_t bytes = (size_t)B * S * sizeof(int32_t);
+  QZO_CUDA_TRY(cudaMemcpyAsync(m->tok_dev, h_tokens, bytes, cudaMemcpyHostToDevice, m->stream));
+  QZO_CUDA_TRY(cudaMemcpyAsync(m->lab_dev, h_labels, bytes, cudaMemcpyHostToDevice, m->stream));
+  return step_device(m, m->tok_dev, m->lab_dev, B, S, seed, eps, lr, clip, h_out);
+}
+
+int qzo_debug_set_capture(qzo_model* m, int layer) {
+  if (!m || layer < -1 || layer >= m->desc.n_layers) return QZO_ERR_BAD_ARG;
+  m->capture_layer = layer;
+  return QZO_OK;
+}
+
+int qzo_debug_layer_output(qzo_model* m, int layer, int which, void* d_out, size_t bytes) {
+  if (!m || !d_out || m->last_T <= 0) return QZO_ERR_BAD_ARG;
+  if (which == 0) {
+    if (layer != m->capture_layer) return QZO_ERR_BAD_ARG;
+    const size_t need = (size_t)m->last_T * m->desc.d_model * 2;
+    if (bytes < need) return QZO_ERR_BAD_ARG;
+    QZO_CUDA_TRY(cudaMemcpyAsync(d_out, m->capture, need, cudaMemcpyDeviceToDevice, m->stream));
+  } else if (which == 1) {
+    const size_t need = (size_t)m->last_T * m->desc.vocab * 4;
+    if (bytes < need) return QZO_ERR_BAD_ARG;
+    QZO_CUDA_TRY(cudaMemcpyAsync(d_out, m->logits, need, cudaMemcpyDeviceToDevice, m->stream));
+  } else {
+    return QZO_ERR_BAD_ARG;
+  }
+  return QZO_OK;
+}
+
+int qzo_device_status(qzo_model* m, int* h_status) {
+  if (!m || !h_status) return QZO_ERR_BAD_ARG;
+  QZO_CUDA_TRY(cudaMemcpyAsync(h_status, m->status, sizeof(int), cudaMemcpyDeviceToHost, m->stream));
+  QZO_CUDA_TRY(cudaStreamSynchronize(m->stream));
+  return *h_status ? QZO_ERR_DEVICE_TIMEOUT : QZO_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,42 @@
+// Shared declarations of the library's translation units: error codes, launch checks,
+// small device helpers.  Nothing here is shared with the CPU oracle.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/qzo.h"
+
+namespace qzo {
+
+// Last CUDA error seen by any entry point (per process; see qzo_last_cuda_error).
+void set_last_cuda_error(cudaError_t e);
+
+#define QZO_CUDA_TRY(expr)                                  \
+  do {                                                      \
+    cudaError_t _e = (expr);                                \
+    if (_e != cudaSuccess) {                                \
+      ::qzo::set_last_cuda_error(_e);                       \
+      return QZO_ERR_CUDA;                                  \
+    }                                                       \
+  } while (0)
+
+#define QZO_TRY(expr)                                       \
+  do {                                                      \
+    int _s = (expr);                                        \
+    if (_s != QZO_OK) return _s;                            \
+  } while (0)
+
+constexpr int kGroup = 128;          // rows of one quantisation group (paper: group 128)
+constexpr int kTileN = 128;          // output features per GEMM tile (UMMA M)
+constexpr int kBlockK = 64;          // K elements per pipeline stage (one 128-byte swizzle atom of bf16)
+constexpr int kPackedTileBytes = kTileN * kBlockK / 2;   // 4096: one (n-tile, k-block) of packed nibbles
+
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+inline int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// Checks that the current device is a compute-capability 10.x part; there is no other backend.
+int check_device();
+
+}  // namespace qzo

@@ -1,0 +1,134 @@
+"""GPU parity of the model-level entry points against the oracle on the tiny configurations:
+per-block outputs and logits within 2e-2 (max relative), losses within 1e-3 absolute, updated
+scales within one bf16 ulp given the oracle's clipped d'."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import model as omodel, qzo as oqzo
+from paper_2505_13430_b200 import inputs
+from tests.helpers import build_oracle_model, clone_model
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2505_13430_b200 import qzo
+    return qzo
+
+
+def _relerr(got, ref):
+    got = got.float().cpu().numpy().astype(np.float64)
+    return np.abs(got - ref).max() / np.abs(ref).max()
+
+
+def _setup(lib, name, weight_gain=1.0):
+    cfg = inputs.model_cfg(name)
+    c = inputs.CONFIGS[name]
+    raw = inputs.raw_model_tensors(cfg, seed=1000)
+    if weight_gain != 1.0:
+        for layer in raw["layers"]:
+            for ent in layer["lin"].values():
+                ent["w"] = ent["w"] * weight_gain
+    om = build_oracle_model(raw)
+    gm = lib.build_model_from_raw(raw, c["batch"] * c["seq"])
+    tok, lab = inputs.tokens_and_labels(cfg, c["batch"], c["seq"], seed=7)
+    return cfg, c, om, gm, tok, lab
+
+
+def _bf16_ulp_diff(a, b):
+    def key(t):
+        i = t.view(torch.int16).to(torch.int32) & 0xFFFF
+        return torch.where(i >= 0x8000, 0x8000 - i, i)
+    return (key(a) - key(b)).abs()
+
+
+@pytest.mark.parametrize("name,gain", [("tiny", 1.0), ("tiny", 6.0), ("tiny_opt", 4.0)])
+def test_forward_and_step_match_oracle(lib, name, gain):
+    cfg, c, om, gm, tok, lab = _setup(lib, name, gain)
+    T = c["batch"] * c["seq"]
+    seed, eps, lr, clip = 42, c["eps"], c["lr"], c["clip"]
+    # the library's quantiser produced the same scales as the oracle's (bit-exact)
+    order = omodel.LINEAR_ORDER[cfg["arch"]]
+    for li in range(cfg["n_layers"]):
+        for i, nm in enumerate(order):
+            assert np.array_equal(gm.scales_of(li, i).float().cpu().numpy(), om["layers"][li]["lin"][nm]["s"])
+    tok_d, lab_d = tok.cuda(), lab.cuda()
+    losses = {}
+    for sign in (+1, -1, 0):
+        cap = {}
+        ref_loss = omodel.forward_loss(om, tok.numpy(), lab.numpy(), seed, sign, eps, capture=cap)
+        for li in range(cfg["n_layers"]):
+            gm.qzo_debug_set_capture(li)
+            loss = float(gm.qzo_forward_loss(tok_d, lab_d, seed, sign, eps).cpu()[0])
+            hid = gm.qzo_debug_layer_output(li, 0, T)
+            assert _relerr(hid, cap["hidden"][li]) <= 2e-2, (sign, li)
+        logits = gm.qzo_debug_layer_output(0, 1, T)
+        assert _relerr(logits, cap["logits"]) <= 2e-2
+        assert abs(loss - ref_loss) <= 1e-3, (sign, loss, ref_loss)
+        losses[sign] = (loss, ref_loss)
+    assert gm.qzo_device_status() == 0
+    # run-to-run determinism of the loss
+    l1 = gm.qzo_forward_loss(tok_d, lab_d, seed, +1, eps).cpu().clone()
+    l2 = gm.qzo_forward_loss(tok_d, lab_d, seed, +1, eps).cpu().clone()
+    assert torch.equal(l1.view(torch.int32), l2.view(torch.int32))
+
+    # update with the oracle's clipped d': scales within one bf16 ulp
+    d_ref = oqzo.directional_derivative(losses[+1][1], losses[-1][1], eps)
+    dc_ref = oqzo.ddc_clip(d_ref, clip)
+    before = gm.scales.clone()
+    gm.qzo_update_scales(seed, lr * 50, dc_ref, clip)        # larger lr so that most scales move
+    om2 = clone_model(om)
+    oqzo.update_model_scales(om2, seed, lr * 50, dc_ref)
+    moved = 0
+    for li in range(cfg["n_layers"]):
+        for i, nm in enumerate(order):
+            got = gm.scales_of(li, i).cpu()
+            ref = torch.from_numpy(om2["layers"][li]["lin"][nm]["s"]).bfloat16()
+            assert int(_bf16_ulp_diff(got, ref).max()) <= 1
+            moved += int((got != torch.from_numpy(om["layers"][li]["lin"][nm]["s"]).bfloat16()).sum())
+    assert moved > 0 or dc_ref == 0.0
+    gm.scales.copy_(before)
+
+    # whole step through the C ABI (device tokens and host tokens): same losses, d from them, d' clipped
+    lp, lm, d, dc = gm.qzo_step(tok_d, lab_d, seed, eps, lr, clip)
+    assert abs(lp - losses[+1][1]) <= 1e-3 and abs(lm - losses[-1][1]) <= 1e-3
+    assert abs(d - (np.float32(lp) - np.float32(lm)) / np.float32(2 * eps)) <= 1e-3 * max(1.0, abs(d))
+    assert dc == min(max(d, -clip), clip)
+    after_dev = gm.scales.clone()
+    gm.scales.copy_(before)
+    lp2, lm2, d2, dc2 = gm.qzo_step_host(tok.contiguous(), lab.contiguous(), seed, eps, lr, clip)
+    assert (lp2, lm2, d2, dc2) == (lp, lm, d, dc)
+    assert torch.equal(gm.scales.view(torch.int16), after_dev.view(torch.int16))
+    # the step's update equals the standalone update with the step's own d'
+    gm.scales.copy_(before)
+    gm.qzo_update_scales(seed, lr, d, clip)
+    assert torch.equal(gm.scales.view(torch.int16), after_dev.view(torch.int16))
+    # C = 0: d' = 0 and the scales stay bit-identical
+    gm.scales.copy_(before)
+    out = gm.qzo_step(tok_d, lab_d, seed, eps, lr, 0.0)
+    assert out[3] == 0.0 and torch.equal(gm.scales.view(torch.int16), before.view(torch.int16))
+    gm.close()
+
+
+def test_batch_limits_and_bad_arguments(lib):
+    cfg, c, om, gm, tok, lab = _setup(lib, "tiny")
+    tok_d, lab_d = tok.cuda(), lab.cuda()
+    with pytest.raises(lib.QzoError) as e:
+        gm.qzo_forward_loss(tok_d, lab_d, 1, 2, 1e-3)
+    assert e.value.status == lib.ERR_BAD_ARG
+    big = torch.zeros((8, 64), dtype=torch.int32, device="cuda")
+    with pytest.raises(lib.QzoError) as e:
+        gm.qzo_forward_loss(big, big, 1, 1, 1e-3)
+    assert e.value.status == lib.ERR_WORKSPACE
+    with pytest.raises(lib.QzoError) as e:
+        gm.qzo_update_scales(1, 1e-5, float("inf"), 100.0)
+    assert e.value.status == lib.ERR_NONFINITE
+    # a smaller batch than the maximum works, and ignored labels do not count
+    small_tok, small_lab = tok_d[:2, :33].contiguous(), lab_d[:2, :33].contiguous()
+    small_lab[:, -1] = -100
+    loss = float(gm.qzo_forward_loss(small_tok, small_lab, 3, 0, 1e-3).cpu()[0])
+    ref = omodel.forward_loss(om, small_tok.cpu().numpy(), small_lab.cpu().numpy(), 3, 0, 1e-3)
+    assert abs(loss - ref) <= 1e-3
+    gm.close()
