@@ -1,0 +1,265 @@
+#!/usr/bin/env python
+"""Benchmark of the QZO hot path: whole optimisation steps (two perturbed forwards + seeded
+scale update) on a synthetic int4 Llama-2-7B-shaped model, one B200 per rank.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+Prints ONE JSON line (rank 0).  `value` is steps/s with tokens already resident on the device;
+`e2e` is the same step through the host-buffer entry point (token upload and loss read-back
+inside the timed region).  `--impl reference` times the CPU oracle on a bounded sample.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        self.gpu = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=self.file, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.file:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        os.unlink(self.file.name)
+        if sm:
+            sm.sort()
+            out = {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+        return out
+
+
+def oracle_sample(workload, n_seq=2):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload: ONE decoder block's
+    forward (one perturbation sign) on n_seq sequences, extrapolated to a whole step by
+    x n_layers x 2 signs x (batch / n_seq).  Returns (steps_per_s, cores, description)."""
+    import numpy as np
+    import torch
+    from oracle import int4, model as omodel
+    from paper_2505_13430_b200 import inputs
+    c = inputs.CONFIGS[workload]
+    cfg = inputs.model_cfg(workload, n_layers=1)
+    raw = inputs.raw_model_tensors(cfg, seed=1000)
+    m = {"cfg": dict(cfg), "embed": raw["embed"].float().numpy(), "lm_head": raw["lm_head"].float().numpy()[:8],
+         "final_norm_w": raw["final_norm_w"].numpy()}
+    if "pos_embed" in raw:
+        m["pos_embed"] = raw["pos_embed"].float().numpy()
+        m["final_norm_b"] = raw["final_norm_b"].numpy()
+    layer = {k: v.float().numpy() for k, v in raw["layers"][0].items() if k != "lin"}
+    layer["lin"] = {}
+    for name, ent in raw["layers"][0]["lin"].items():
+        q, s = int4.quantize_int4(ent["w"].numpy())
+        layer["lin"][name] = {"q": q, "s": s}
+        if "bias" in ent:
+            layer["lin"][name]["bias"] = ent["bias"].numpy()
+    m["layers"] = [layer]
+    del raw
+    n_seq = min(n_seq, c["batch"])
+    tok, lab = inputs.tokens_and_labels(cfg, n_seq, c["seq"], seed=7)
+    lab = np.where(lab.numpy() >= 8, -100, lab.numpy())       # the sample keeps 8 rows of the head only
+    t0 = time.perf_counter()
+    omodel.forward_loss(m, tok.numpy(), lab, 42, +1, c["eps"])
+    dt = time.perf_counter() - t0
+    step_s = dt * c["n_layers"] * 2 * (c["batch"] / n_seq)
+    cores = torch.get_num_threads()
+    desc = (f"oracle forward of 1 of {c['n_layers']} decoder blocks, 1 of 2 signs, {n_seq} of {c['batch']} "
+            f"sequences (S={c['seq']}) in {dt:.2f} s; extrapolated linearly to a whole step")
+    return 1.0 / step_s, cores, desc
+
+
+def run_reference(args, workload):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals = []
+    cores, desc = 0, ""
+    for i in range(args.warmup + args.steps):
+        v, cores, desc = oracle_sample(workload, n_seq=1)
+        if i >= args.warmup:
+            vals.append(v)
+    value = sum(vals) / len(vals)
+    c = bench_config(workload, args.gpus)
+    line = {"impl": "reference", "metric": "qzo_steps_per_s", "value": value, "unit": "steps/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1000.0 / value, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": c,
+            "cpu_baseline": {"value": value, "unit": "steps/s", "cores": cores, "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def bench_config(workload, n_gpus):
+    from paper_2505_13430_b200 import inputs
+    c = inputs.CONFIGS[workload]
+    return {"workload": f"{workload}: {c['arch']}-shaped random-init int4 model, {c['n_layers']} layers, d={c['d_model']}, "
+                        f"{c['n_heads']} heads, FFN {c['d_ffn']}, vocab {c['vocab']}, group-128 bf16 scales; full QZO step "
+                        f"(2 perturbed forwards + seeded scale update)",
+            "batch_per_gpu": c["batch"], "seq_len": c["seq"], "eps": c["eps"], "lr": c["lr"], "clip": c["clip"],
+            "parallelism": f"{n_gpus} independent replica(s), no collective",
+            "l2": "inputs larger than L2: every step streams 3.3 GB+ of int4 weights"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama7b")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+    workload = args.workload
+
+    if args.impl == "reference":
+        run_reference(args, workload)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2505_13430_b200 import inputs, qzo
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    c = inputs.CONFIGS[workload]
+    cfg = inputs.model_cfg(workload)
+    B, S = c["batch"], c["seq"]
+    model = qzo.build_random_model_gpu(cfg, B * S, seed=1000 + rank)
+    tok, lab = inputs.tokens_and_labels(cfg, B, S, seed=7 + rank)
+    tok_pin, lab_pin = tok.contiguous().pin_memory(), lab.contiguous().pin_memory()
+    tok_d, lab_d = tok.cuda(), lab.cuda()
+    n_gemm = cfg["n_layers"] * len(inputs.linear_shapes(cfg)) * 2
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        ev0.record(stream)
+        for t in range(steps):
+            fn(t)
+        ev1.record(stream)
+        barrier()
+        ms = ev0.elapsed_time(ev1)
+        if world > 1:
+            tt = torch.tensor([ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            ms = float(tt.item())
+        return ms
+
+    seed0 = 42
+    for t in range(args.warmup):
+        model.qzo_step(tok_d, lab_d, seed0 + t, c["eps"], c["lr"], c["clip"], read_back=False)
+    model.qzo_profile_gemms(n_gemm * args.steps)
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = qzo.qzo_launch_count()
+    ms = timed(lambda t: model.qzo_step(tok_d, lab_d, seed0 + 100 + t, c["eps"], c["lr"], c["clip"], read_back=False),
+               args.steps)
+    launches = qzo.qzo_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    n_l, gemm_ms, gemm_flops = model.qzo_profile_read()
+    model.qzo_profile_gemms(0)
+    status = model.qzo_device_status()
+    if status != 0:
+        raise SystemExit("device status word set: a bounded wait expired during the benchmark")
+
+    # end to end: host (pinned) tokens in, losses out, every step
+    for t in range(2):
+        model.qzo_step_host(tok_pin, lab_pin, seed0 + t, c["eps"], c["lr"], c["clip"])
+    e2e_ms = timed(lambda t: model.qzo_step_host(tok_pin, lab_pin, seed0 + 200 + t, c["eps"], c["lr"], c["clip"]),
+                   args.steps)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    value = world * args.steps / (ms / 1000.0)
+    e2e = world * args.steps / (e2e_ms / 1000.0)
+    achieved = gemm_flops / (gemm_ms / 1000.0) / 1e12 if gemm_ms > 0 else 0.0
+    peak = peaks["bf16_tflops_sustained"]
+    line = {"metric": "qzo_steps_per_s", "value": value, "unit": "steps/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": bench_config(workload, world),
+            "clocks": clocks,
+            "e2e": {"value": e2e, "unit": "steps/s", "h2d_bytes_per_step": 2 * B * S * 4, "d2h_bytes_per_step": 16},
+            "gpu_launches": int(launches),
+            "roofline": {"kernel": "w4a16_gemm_kernel (perturbed W4A16 GEMM, all block linears)", "bound": "tensor",
+                         "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                         "peak_source": f"{peaks['source']} bf16 sustained", "traffic": None,
+                         "launches": int(n_l), "gemm_share_of_step": gemm_ms / ms if ms > 0 else None}}
+    if not args.no_cpu_baseline:
+        v, cores, desc = oracle_sample(workload)
+        line["cpu_baseline"] = {"value": v, "unit": "steps/s", "cores": cores, "kind": "oracle", "sample": desc}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -194,6 +194,13 @@ int qzo_debug_layer_output(qzo_model* m, int layer, int which, void* d_out, size
 /* Reads the device status word (0 = no bounded wait has expired since init). Synchronises. */
 int qzo_device_status(qzo_model* m, int* h_status);
 
+/* Per-GEMM timing: with max_launches > 0 every later perturbed-GEMM launch of this model (up to
+ * max_launches between two reads) is bracketed by a pair of CUDA events on the model's stream;
+ * 0 switches it off.  qzo_profile_read synchronises, returns the number of bracketed launches,
+ * the sum of their durations in ms and of their algorithmic FLOPs (2 M K N), and rearms. */
+int qzo_profile_gemms(qzo_model* m, int max_launches);
+int qzo_profile_read(qzo_model* m, int64_t* launches, double* total_ms, double* total_flops);
+
 /* Number of kernels the library launched since the process started (for benchmark accounting). */
 int64_t qzo_launch_count(void);
 

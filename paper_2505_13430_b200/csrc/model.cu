@@ -117,6 +117,11 @@ struct qzo_model {
   int* status = nullptr;
   int capture_layer = -1;
   int last_T = 0;
+  // optional per-GEMM timing (CUDA events around every perturbed GEMM launch)
+  bool profiling = false;
+  std::vector<cudaEvent_t> events;
+  size_t events_used = 0;
+  double profiled_flops = 0.0;
 };
 
 namespace qzo {
@@ -159,15 +164,23 @@ int plan_workspace(const qzo_model_desc& d, int T, WsPlan* p) {
   return QZO_OK;
 }
 
-static int norm(const qzo_model* m, const __nv_bfloat16* in, const float* w, const float* b, int T, __nv_bfloat16* out) {
+static int norm(qzo_model* m, const __nv_bfloat16* in, const float* w, const float* b, int T, __nv_bfloat16* out) {
   if (m->desc.arch == QZO_ARCH_LLAMA) return launch_rmsnorm(in, w, m->desc.norm_eps, T, m->desc.d_model, out, m->stream);
   return launch_layernorm(in, w, b, m->desc.norm_eps, T, m->desc.d_model, out, m->stream);
 }
 
-static int linear(const qzo_model* m, const Linear& L, const __nv_bfloat16* in, const __nv_bfloat16* residual,
+static int linear(qzo_model* m, const Linear& L, const __nv_bfloat16* in, const __nv_bfloat16* residual,
                   __nv_bfloat16* out, int ldo, int T, uint64_t seed, int sign, float eps) {
-  return launch_perturbed_gemm(in, L.wq, m->scales + L.idx_base, L.bias, residual, out, ldo, T, L.K, L.N, seed,
-                               (uint64_t)L.idx_base, sign, eps, m->gemm_ws, m->gemm_ws_bytes, m->status, m->stream);
+  const bool timed = m->profiling && m->events_used + 2 <= m->events.size();
+  if (timed) QZO_CUDA_TRY(cudaEventRecord(m->events[m->events_used], m->stream));
+  QZO_TRY(launch_perturbed_gemm(in, L.wq, m->scales + L.idx_base, L.bias, residual, out, ldo, T, L.K, L.N, seed,
+                                (uint64_t)L.idx_base, sign, eps, m->gemm_ws, m->gemm_ws_bytes, m->status, m->stream));
+  if (timed) {
+    QZO_CUDA_TRY(cudaEventRecord(m->events[m->events_used + 1], m->stream));
+    m->events_used += 2;
+    m->profiled_flops += 2.0 * T * (double)L.K * (double)L.N;
+  }
+  return QZO_OK;
 }
 
 int forward_loss(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S, uint64_t seed, int sign,
@@ -456,8 +469,41 @@ int qzo_init_model(const qzo_model_desc* desc, const qzo_tensor* tensors, int n_
   return QZO_OK;
 }
 
+int qzo_profile_gemms(qzo_model* m, int max_launches) {
+  if (!m || max_launches < 0) return QZO_ERR_BAD_ARG;
+  for (cudaEvent_t e : m->events) cudaEventDestroy(e);
+  m->events.clear();
+  m->events_used = 0;
+  m->profiled_flops = 0.0;
+  m->profiling = max_launches > 0;
+  for (int i = 0; i < 2 * max_launches; ++i) {
+    cudaEvent_t e;
+    QZO_CUDA_TRY(cudaEventCreate(&e));
+    m->events.push_back(e);
+  }
+  return QZO_OK;
+}
+
+int qzo_profile_read(qzo_model* m, int64_t* launches, double* total_ms, double* total_flops) {
+  if (!m || !launches || !total_ms || !total_flops) return QZO_ERR_BAD_ARG;
+  QZO_CUDA_TRY(cudaStreamSynchronize(m->stream));
+  double ms = 0.0;
+  for (size_t i = 0; i + 1 < m->events_used; i += 2) {
+    float t = 0.0f;
+    QZO_CUDA_TRY(cudaEventElapsedTime(&t, m->events[i], m->events[i + 1]));
+    ms += t;
+  }
+  *launches = (int64_t)(m->events_used / 2);
+  *total_ms = ms;
+  *total_flops = m->profiled_flops;
+  m->events_used = 0;
+  m->profiled_flops = 0.0;
+  return QZO_OK;
+}
+
 int qzo_free_model(qzo_model* m) {
   if (!m) return QZO_ERR_BAD_ARG;
+  for (cudaEvent_t e : m->events) cudaEventDestroy(e);
   delete m;
   return QZO_OK;
 }

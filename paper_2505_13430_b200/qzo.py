@@ -26,7 +26,7 @@ EXPORTS = (
     "qzo_gemm_workspace_bytes", "qzo_perturbed_gemm", "qzo_update_scales_flat", "qzo_num_scales",
     "qzo_scale_layout", "qzo_workspace_bytes", "qzo_init_model", "qzo_free_model", "qzo_forward_loss",
     "qzo_update_scales", "qzo_step", "qzo_step_host", "qzo_debug_set_capture", "qzo_debug_layer_output",
-    "qzo_device_status", "qzo_launch_count",
+    "qzo_device_status", "qzo_launch_count", "qzo_profile_gemms", "qzo_profile_read",
 )
 
 
@@ -85,6 +85,8 @@ def _load():
         "qzo_debug_set_capture": (ci, [vp, ci]),
         "qzo_debug_layer_output": (ci, [vp, ci, ci, vp, sz]),
         "qzo_device_status": (ci, [vp, P(ci)]),
+        "qzo_profile_gemms": (ci, [vp, ci]),
+        "qzo_profile_read": (ci, [vp, P(i64), P(ctypes.c_double), P(ctypes.c_double)]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -315,6 +317,16 @@ class Model:
             _check(rc, "qzo_device_status")
         return st.value
 
+    def qzo_profile_gemms(self, max_launches):
+        _check(_lib.qzo_profile_gemms(self.handle, max_launches), "qzo_profile_gemms")
+
+    def qzo_profile_read(self):
+        """-> (launches, total_ms, total_flops) of the bracketed GEMM launches since the last read."""
+        n, ms, fl = ctypes.c_int64(0), ctypes.c_double(0), ctypes.c_double(0)
+        _check(_lib.qzo_profile_read(self.handle, ctypes.byref(n), ctypes.byref(ms), ctypes.byref(fl)),
+               "qzo_profile_read")
+        return n.value, ms.value, fl.value
+
     def scales_of(self, layer, linear):
         """View of one linear's scales [G][N] inside the flat buffer."""
         base, G, N = qzo_scale_layout(self.cfg, layer, linear)
@@ -353,3 +365,45 @@ def build_model_from_raw(raw, max_tokens, quantized=None):
             if "bias" in ent:
                 t[f"L{li}.{name}.bias"] = ent["bias"].float().cuda()
     return Model(cfg, t, max_tokens)
+
+
+def build_random_model_gpu(cfg, max_tokens, seed=1000):
+    """Random-init int4 model generated and quantised tensor by tensor on the device
+    (fp32 N(0, 0.02) weights -> library quantiser), so that no full-precision copy of the
+    model ever exists.  Used by the benchmark for the large configurations."""
+    from .inputs import linear_shapes, normal_fp32
+    flat, _ = qzo_num_scales(cfg)
+    d, V = cfg["d_model"], cfg["vocab"]
+    sid = [int(seed)]
+
+    def nxt():
+        sid[0] += 1
+        return sid[0]
+
+    scales = torch.zeros((flat,), dtype=torch.bfloat16, device="cuda")
+    t = {"embed": normal_fp32((V, d), 0.02, nxt(), "cuda").bfloat16(),
+         "lm_head": normal_fp32((V, d), 0.02, nxt(), "cuda").bfloat16(),
+         "final_norm_w": torch.ones(d, device="cuda"), "scales": scales}
+    opt = cfg["arch"] == "opt"
+    if opt:
+        t["pos_embed"] = normal_fp32((cfg["max_seq"], d), 0.02, nxt(), "cuda").bfloat16()
+        t["final_norm_b"] = torch.zeros(d, device="cuda")
+    for li in range(cfg["n_layers"]):
+        t[f"L{li}.norm1_w"] = torch.ones(d, device="cuda")
+        t[f"L{li}.norm2_w"] = torch.ones(d, device="cuda")
+        if opt:
+            t[f"L{li}.norm1_b"] = torch.zeros(d, device="cuda")
+            t[f"L{li}.norm2_b"] = torch.zeros(d, device="cuda")
+        for idx, (name, K, N) in enumerate(linear_shapes(cfg)):
+            w = normal_fp32((K, N), 0.02, nxt(), "cuda")
+            words, s = qzo_quantize_int4(w)
+            del w
+            base, G, Nn = qzo_scale_layout(cfg, li, idx)
+            scales[base:base + G * Nn] = s.reshape(-1)
+            t[f"L{li}.{name}.qweight"] = words
+            if opt:
+                t[f"L{li}.{name}.bias"] = normal_fp32((N,), 0.02, nxt(), "cuda")
+    m = Model(cfg, t, max_tokens)
+    del t
+    torch.cuda.empty_cache()
+    return m
