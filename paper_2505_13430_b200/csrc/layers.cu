@@ -133,44 +133,160 @@ __global__ void rope_kernel(__nv_bfloat16* __restrict__ q, __nv_bfloat16* __rest
   }
 }
 
-// Causal attention, one warp per (batch, head, query): online softmax over keys 0..query.
-// DH in {64, 128}; each lane holds DH/32 features.
+// Causal attention with online softmax on the legacy tensor-core path (mma.sync m16n8k16,
+// bf16 in, fp32 accumulate).  One CTA = 64 queries of one (batch, head); each of the four
+// warps owns 16 query rows; keys are walked in blocks of 64 up to the diagonal block.
+// Attention is ~0.5 % of a step's FLOPs, so it stays off the tcgen05 path.
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16_16816(float c[4], const uint32_t a[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
 template <int DH>
-__global__ void attention_simple_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
-                                        const __nv_bfloat16* __restrict__ v, int ldq, int ldk, int ldv,
-                                        __nv_bfloat16* __restrict__ out, int ldo, int B, int S, int H, float scale) {
-  constexpr int E = DH / 32;
-  const int64_t wid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int lane = threadIdx.x & 31;
-  if (wid >= (int64_t)B * H * S) return;
-  const int sq = (int)(wid % S);
-  const int h = (int)((wid / S) % H);
-  const int b = (int)(wid / ((int64_t)S * H));
-  const int t = b * S + sq;
-  float qv[E], acc[E];
+__global__ void __launch_bounds__(128)
+attention_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+                     const __nv_bfloat16* __restrict__ v, int ldq, int ldk, int ldv,
+                     __nv_bfloat16* __restrict__ out, int ldo, int S, float scale_log2e) {
+  constexpr int BQ = 64, BK = 64;
+  constexpr int LD = DH + 8;                       // padded row (bf16 elements): conflict-free ldmatrix
+  extern __shared__ __align__(16) uint8_t att_smem[];
+  __nv_bfloat16* sQ = reinterpret_cast<__nv_bfloat16*>(att_smem);
+  __nv_bfloat16* sK = sQ + BQ * LD;
+  __nv_bfloat16* sV = sK + BK * LD;
+
+  const int qb = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t4 = lane & 3;
+  const size_t tok_base = (size_t)b * S;
+  const int q0 = qb * BQ;
+
+  // stage a [64][DH] tile (rows beyond S are zero)
+  auto load_tile = [&](__nv_bfloat16* dst, const __nv_bfloat16* src, int ld, int row0) {
+    constexpr int CH = DH / 8;                     // 16-byte chunks per row
+    for (int i = threadIdx.x; i < 64 * CH; i += 128) {
+      const int r = i / CH, c = i % CH;
+      uint4 val = make_uint4(0, 0, 0, 0);
+      if (row0 + r < S) val = *reinterpret_cast<const uint4*>(src + (tok_base + row0 + r) * ld + h * DH + c * 8);
+      *reinterpret_cast<uint4*>(dst + r * LD + c * 8) = val;
+    }
+  };
+  load_tile(sQ, q, ldq, q0);
+  __syncthreads();
+
+  // Q fragments of this warp's 16 rows, all of DH
+  uint32_t qf[DH / 16][4];
+  {
+    const int row = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
 #pragma unroll
-  for (int e = 0; e < E; ++e) {
-    qv[e] = __bfloat162float(q[(size_t)t * ldq + h * DH + lane * E + e]) * scale;
-    acc[e] = 0.0f;
+    for (int kk = 0; kk < DH / 16; ++kk) {
+      const int col = kk * 16 + (lane >> 4) * 8;
+      ldmatrix_x4((uint32_t)__cvta_generic_to_shared(sQ + row * LD + col), qf[kk][0], qf[kk][1], qf[kk][2], qf[kk][3]);
+    }
   }
-  float m = -INFINITY, l = 0.0f;
-  for (int j = 0; j <= sq; ++j) {
-    const size_t tk = (size_t)(b * S + j);
-    float part = 0.0f;
+  float o[DH / 8][4];
 #pragma unroll
-    for (int e = 0; e < E; ++e) part += qv[e] * __bfloat162float(k[tk * ldk + h * DH + lane * E + e]);
-    const float sc = warp_sum(part);
-    const float mn = fmaxf(m, sc);
-    const float corr = __expf(m - mn);
-    const float pj = __expf(sc - mn);
-    l = l * corr + pj;
+  for (int i = 0; i < DH / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.0f;
+  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.0f, l1 = 0.0f;      // rows g and g + 8 of the warp's 16
+  const int qrow0 = q0 + warp * 16 + g, qrow1 = qrow0 + 8;
+
+  for (int kb = 0; kb <= qb; ++kb) {
+    __syncthreads();                                // previous K/V tiles fully consumed
+    load_tile(sK, k, ldk, kb * BK);
+    load_tile(sV, v, ldv, kb * BK);
+    __syncthreads();
+
+    // scores: 16 x 64 per warp
+    float sc[BK / 8][4];
 #pragma unroll
-    for (int e = 0; e < E; ++e) acc[e] = acc[e] * corr + pj * __bfloat162float(v[tk * ldv + h * DH + lane * E + e]);
-    m = mn;
+    for (int j = 0; j < BK / 8; ++j) sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.0f;
+#pragma unroll
+    for (int kk = 0; kk < DH / 16; ++kk) {
+#pragma unroll
+      for (int jp = 0; jp < BK / 16; ++jp) {        // two n8 tiles (16 keys) per ldmatrix.x4
+        uint32_t b00, b01, b10, b11;
+        const int key = jp * 16 + (lane & 7) + (lane >> 4) * 8;
+        const int col = kk * 16 + ((lane >> 3) & 1) * 8;
+        ldmatrix_x4((uint32_t)__cvta_generic_to_shared(sK + key * LD + col), b00, b01, b10, b11);
+        mma_bf16_16816(sc[2 * jp], qf[kk], b00, b01);
+        mma_bf16_16816(sc[2 * jp + 1], qf[kk], b10, b11);
+      }
+    }
+    // causal mask (only the diagonal block can cross it)
+    if (kb == qb) {
+#pragma unroll
+      for (int j = 0; j < BK / 8; ++j) {
+        const int key = kb * BK + j * 8 + 2 * t4;
+        if (key > qrow0) sc[j][0] = -INFINITY;
+        if (key + 1 > qrow0) sc[j][1] = -INFINITY;
+        if (key > qrow1) sc[j][2] = -INFINITY;
+        if (key + 1 > qrow1) sc[j][3] = -INFINITY;
+      }
+    }
+    // online softmax (base-2 exponent with the 1/sqrt(dh) scale folded in)
+    float mx0 = m0, mx1 = m1;
+#pragma unroll
+    for (int j = 0; j < BK / 8; ++j) {
+      mx0 = fmaxf(mx0, fmaxf(sc[j][0], sc[j][1]));
+      mx1 = fmaxf(mx1, fmaxf(sc[j][2], sc[j][3]));
+    }
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+    const float corr0 = exp2f((m0 - mx0) * scale_log2e), corr1 = exp2f((m1 - mx1) * scale_log2e);
+    m0 = mx0; m1 = mx1;
+    float rs0 = 0.0f, rs1 = 0.0f;
+    uint32_t pf[BK / 16][4];
+#pragma unroll
+    for (int j = 0; j < BK / 8; ++j) {
+      const float p0 = exp2f((sc[j][0] - mx0) * scale_log2e), p1 = exp2f((sc[j][1] - mx0) * scale_log2e);
+      const float p2 = exp2f((sc[j][2] - mx1) * scale_log2e), p3 = exp2f((sc[j][3] - mx1) * scale_log2e);
+      rs0 += p0 + p1; rs1 += p2 + p3;
+      pf[j >> 1][(j & 1) * 2] = pack_bf16x2(p0, p1);
+      pf[j >> 1][(j & 1) * 2 + 1] = pack_bf16x2(p2, p3);
+    }
+    l0 = l0 * corr0 + rs0; l1 = l1 * corr1 + rs1;
+#pragma unroll
+    for (int i = 0; i < DH / 8; ++i) { o[i][0] *= corr0; o[i][1] *= corr0; o[i][2] *= corr1; o[i][3] *= corr1; }
+    // O += P V
+#pragma unroll
+    for (int kk = 0; kk < BK / 16; ++kk) {
+#pragma unroll
+      for (int np = 0; np < DH / 16; ++np) {        // two n8 tiles of the head dimension per ldmatrix.x4.trans
+        uint32_t b00, b01, b10, b11;
+        const int key = kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+        const int col = np * 16 + (lane >> 4) * 8;
+        ldmatrix_x4_trans((uint32_t)__cvta_generic_to_shared(sV + key * LD + col), b00, b01, b10, b11);
+        mma_bf16_16816(o[2 * np], pf[kk], b00, b01);
+        mma_bf16_16816(o[2 * np + 1], pf[kk], b10, b11);
+      }
+    }
   }
-  const float inv = 1.0f / l;
+  // normalise and store
+  l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+  l1 += __shfl_xor_sync(0xffffffffu, l1, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+  const float inv0 = 1.0f / l0, inv1 = 1.0f / l1;
 #pragma unroll
-  for (int e = 0; e < E; ++e) out[(size_t)t * ldo + h * DH + lane * E + e] = __float2bfloat16_rn(acc[e] * inv);
+  for (int i = 0; i < DH / 8; ++i) {
+    const int col = h * DH + i * 8 + 2 * t4;
+    if (qrow0 < S)
+      *reinterpret_cast<uint32_t*>(out + (tok_base + qrow0) * ldo + col) = pack_bf16x2(o[i][0] * inv0, o[i][1] * inv0);
+    if (qrow1 < S)
+      *reinterpret_cast<uint32_t*>(out + (tok_base + qrow1) * ldo + col) = pack_bf16x2(o[i][2] * inv1, o[i][3] * inv1);
+  }
 }
 
 // act = silu(gate) * up
@@ -264,13 +380,19 @@ int launch_rope(__nv_bfloat16* q, __nv_bfloat16* k, int ldq, int ldk, const floa
 }
 int launch_attention(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v, int ldq, int ldk, int ldv,
                      __nv_bfloat16* out, int ldo, int B, int S, int H, int dh, cudaStream_t st) {
-  const int64_t warps = (int64_t)B * H * S;
-  const float scale = 1.0f / sqrtf((float)dh);
-  const dim3 grid((unsigned)ceil_div64(warps * 32, 256));
+  const float scale_log2e = 1.4426950408889634f / sqrtf((float)dh);
+  const dim3 grid(ceil_div(S, 64), H, B);
+  if ((ldq % 8) || (ldk % 8) || (ldv % 8) || (ldo % 2)) return QZO_ERR_BAD_ARG;
   if (dh == 64) {
-    QZO_LAUNCH(attention_simple_kernel<64>, grid, dim3(256), 0, st, q, k, v, ldq, ldk, ldv, out, ldo, B, S, H, scale);
+    constexpr int smem = 3 * 64 * (64 + 8) * 2;
+    static bool cfg = false;
+    if (!cfg) { QZO_CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)); cfg = true; }
+    QZO_LAUNCH(attention_mma_kernel<64>, grid, dim3(128), smem, st, q, k, v, ldq, ldk, ldv, out, ldo, S, scale_log2e);
   } else if (dh == 128) {
-    QZO_LAUNCH(attention_simple_kernel<128>, grid, dim3(256), 0, st, q, k, v, ldq, ldk, ldv, out, ldo, B, S, H, scale);
+    constexpr int smem = 3 * 64 * (128 + 8) * 2;
+    static bool cfg = false;
+    if (!cfg) { QZO_CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)); cfg = true; }
+    QZO_LAUNCH(attention_mma_kernel<128>, grid, dim3(128), smem, st, q, k, v, ldq, ldk, ldv, out, ldo, S, scale_log2e);
   } else {
     return QZO_ERR_BAD_ARG;
   }

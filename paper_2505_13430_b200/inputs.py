@@ -17,6 +17,10 @@ CONFIGS = {
     "tiny_opt": dict(arch="opt", n_layers=2, d_model=256, n_heads=4, d_ffn=1024, vocab=1000,
                      max_seq=64, norm_eps=1e-5, rope_theta=0.0, batch=4, seq=48,
                      eps=1e-3, lr=1e-5, clip=10.0),
+    # Tiny variant with head dimension 128 and several ragged attention blocks (parity tests).
+    "tiny_dh128": dict(arch="llama", n_layers=2, d_model=256, n_heads=2, d_ffn=688, vocab=1024,
+                       max_seq=200, norm_eps=1e-5, rope_theta=10000.0, batch=2, seq=200,
+                       eps=1e-3, lr=1e-5, clip=100.0),
     "llama7b": dict(arch="llama", n_layers=32, d_model=4096, n_heads=32, d_ffn=11008,
                     vocab=32000, max_seq=256, norm_eps=1e-5, rope_theta=10000.0,
                     batch=16, seq=256, eps=1e-3, lr=1e-5, clip=100.0),

@@ -44,7 +44,7 @@ def _bf16_ulp_diff(a, b):
     return (key(a) - key(b)).abs()
 
 
-@pytest.mark.parametrize("name,gain", [("tiny", 1.0), ("tiny", 3.0), ("tiny_opt", 1.0), ("tiny_opt", 3.0)])
+@pytest.mark.parametrize("name,gain", [("tiny", 1.0), ("tiny", 3.0), ("tiny_opt", 1.0), ("tiny_opt", 3.0), ("tiny_dh128", 3.0)])
 def test_forward_and_step_match_oracle(lib, name, gain):
     cfg, c, om, gm, tok, lab = _setup(lib, name, gain)
     T = c["batch"] * c["seq"]
