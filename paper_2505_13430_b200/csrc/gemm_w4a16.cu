@@ -31,7 +31,9 @@ namespace qzo {
 
 namespace {
 
-constexpr int kStages = 4;            // pipeline depth over k-blocks
+constexpr int kStagesDequant = 6;     // pipeline depth over k-blocks, int4 path (A operand lives in TMEM)
+constexpr int kStagesBf16 = 4;        // bf16-weight path (A operand tile in shared memory)
+constexpr int kATmemColsPerStage = kBlockK / 2;   // 64 bf16 along K = 32 TMEM columns of 32 bits
 constexpr int kScaleSlots = 4;        // ring of perturbed-scale rows (one per quantisation group)
 constexpr int kNumScaleWarps = 2;
 constexpr int kNumDeqWarps = 8;
@@ -98,9 +100,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
   }
 }
-__device__ __forceinline__ void fence_proxy_async_smem() {
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
@@ -136,6 +135,24 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint6
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// Same MMA with the A operand read from tensor memory (lane = row, 2 bf16 per 32-bit column).
+__device__ __forceinline__ void umma_bf16_tmem_a(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
+                                                 uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t v[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+      ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+        "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+      : "memory");
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -168,13 +185,15 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16(int m, int n) {
 }
 
 // ----------------------------------------------------------------------------- shared memory plan
-template <int TOK>
+template <int TOK, bool DEQUANT>
 struct SmemPlan {
+  static constexpr int kStages = DEQUANT ? kStagesDequant : kStagesBf16;
   static constexpr int kXTileBytes = TOK * kBlockK * 2;
-  static constexpr int kStageBytes = kWTileBytes + kXTileBytes + kPackedTileBytes;
-  static constexpr int kOffW = 0;
-  static constexpr int kOffX = kWTileBytes;
-  static constexpr int kOffP = kWTileBytes + kXTileBytes;
+  // int4 path: [X tile | packed nibbles]; bf16 path: [W tile | X tile]
+  static constexpr int kStageBytes = DEQUANT ? (kXTileBytes + kPackedTileBytes) : (kWTileBytes + kXTileBytes);
+  static constexpr int kOffW = 0;                                   // bf16 path only
+  static constexpr int kOffX = DEQUANT ? 0 : kWTileBytes;
+  static constexpr int kOffP = kXTileBytes;                         // int4 path only
   static constexpr int kOffRaw = kStages * kStageBytes;
   static constexpr int kOffCooked = kOffRaw + kScaleSlots * kRawScaleBytes;
   static constexpr int kOffBars = kOffCooked + kScaleSlots * kCookedScaleBytes;
@@ -191,7 +210,8 @@ template <int TOK, bool DEQUANT, int OUT_MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                   const GemmParams p) {
-  using Plan = SmemPlan<TOK>;
+  using Plan = SmemPlan<TOK, DEQUANT>;
+  constexpr int kStages = Plan::kStages;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* const smem = smem_raw + (base - smem_u32(smem_raw));
@@ -218,7 +238,12 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
   const int kb_end = min(kb_begin + p.kb_per_split, p.num_kb);
   const int nkb = kb_end - kb_begin;                     // >= 1 by construction of the grid
 
-  constexpr uint32_t kTmemCols = TOK < 32 ? 32 : TOK;
+  // TMEM columns: accumulator [0, TOK), then (int4 path) one 32-column A tile per stage
+  constexpr uint32_t kAccCols = TOK < 32 ? 32 : TOK;
+  constexpr uint32_t kUsedCols = DEQUANT ? kAccCols + kStages * kATmemColsPerStage : kAccCols;
+  constexpr uint32_t kTmemCols = kUsedCols <= 32 ? 32 : kUsedCols <= 64 ? 64 : kUsedCols <= 128 ? 128
+                                 : kUsedCols <= 256 ? 256 : 512;
+  static_assert(kUsedCols <= 512, "TMEM budget");
 
   if (threadIdx.x == 0) {
     *abort_flag = 0;
@@ -299,12 +324,19 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         }
         tcgen05_fence_after();
         const uint32_t stage = base + s * Plan::kStageBytes;
-        const uint64_t adesc = umma_desc_k_major_sw128(stage + Plan::kOffW);
         const uint64_t bdesc = umma_desc_k_major_sw128(stage + Plan::kOffX);
+        if (DEQUANT) {
+          const uint32_t a_tmem = tmem_d + kAccCols + (uint32_t)(s * kATmemColsPerStage);
 #pragma unroll
-        for (int k = 0; k < kBlockK / 16; ++k) {
-          umma_bf16(tmem_d, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
-                    (it > 0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < kBlockK / 16; ++k)      // 16 bf16 along K = 8 TMEM columns
+            umma_bf16_tmem_a(tmem_d, a_tmem + (uint32_t)(k * 8), bdesc + (uint64_t)(k * 2), idesc,
+                             (it > 0 || k > 0) ? 1u : 0u);
+        } else {
+          const uint64_t adesc = umma_desc_k_major_sw128(stage + Plan::kOffW);
+#pragma unroll
+          for (int k = 0; k < kBlockK / 16; ++k)
+            umma_bf16(tmem_d, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
+                      (it > 0 || k > 0) ? 1u : 0u);
         }
         umma_commit(bar_empty(s));
       }
@@ -355,7 +387,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     // ------------------------------------------------------------------ de-quantisers, then epilogue
     const int dt = threadIdx.x - kFirstDeqWarp * 32;      // 0..255
     if (DEQUANT) {
-      const int r = dt & (kTileN - 1);                    // row of the tile (output feature)
+      const int r = (warp & 3) * 32 + lane;               // row of the tile = TMEM lane this warp may access
       const int h = dt >> 7;                              // half of the k-block (32 k each)
       const __nv_bfloat162 magic_bias = __halves2bfloat162(__float2bfloat16_rn(136.0f), __float2bfloat16_rn(136.0f));
       __nv_bfloat162 s_hi, s_lo;
@@ -368,38 +400,40 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
           const int gi = it >> 1;
           const int slot = gi % kScaleSlots;
           const uint32_t gph = (uint32_t)(gi / kScaleSlots) & 1u;
-          if (!mbar_wait(bar_sc_full(slot), gph, abort_flag)) { ok = false; break; }
+          if (!__all_sync(0xffffffffu, mbar_wait(bar_sc_full(slot), gph, abort_flag))) { ok = false; break; }
           const uint2 c = *reinterpret_cast<const uint2*>(smem + Plan::kOffCooked + slot * kCookedScaleBytes + r * 8);
           *reinterpret_cast<uint32_t*>(&s_hi) = c.x;
           *reinterpret_cast<uint32_t*>(&s_lo) = c.y;
           mbar_arrive(bar_sc_empty(slot));
         }
         // bar_full(s) completing implies the stage was released by the MMAs that last read it
-        if (!mbar_wait(bar_full(s), ph, abort_flag)) { ok = false; break; }
+        if (!__all_sync(0xffffffffu, mbar_wait(bar_full(s), ph, abort_flag))) { ok = false; break; }
+        tcgen05_fence_after();                              // orders the MMAs' reads of this A stage before the store below
         uint8_t* stage = smem + s * Plan::kStageBytes;
         const uint4 pk = *reinterpret_cast<const uint4*>(stage + Plan::kOffP + (h * kTileN + r) * 16);
         const uint32_t words[4] = {pk.x, pk.y, pk.z, pk.w};
-        uint8_t* row = stage + Plan::kOffW + r * 128;
+        uint32_t outw[16];                                  // k = 32 h + 2 j, 2 j + 1 in register j
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          uint32_t outw[4];
 #pragma unroll
           for (int pp = 0; pp < 4; ++pp) {
             uint32_t x = ((words[i] >> (4 * pp)) & 0x000F000Fu) | 0x43004300u;     // bf16x2 {128 + u_lo, 128 + u_hi}
             __nv_bfloat162 q2 = __hsub2(*reinterpret_cast<__nv_bfloat162*>(&x), magic_bias);   // exact u - 8
             __nv_bfloat162 w2 = __hfma2(q2, s_hi, __hmul2(q2, s_lo));
-            outw[pp] = *reinterpret_cast<uint32_t*>(&w2);
+            outw[i * 4 + pp] = *reinterpret_cast<uint32_t*>(&w2);
           }
-          const int chunk = h * 4 + i;                   // 16-byte chunk along K
-          *reinterpret_cast<uint4*>(row + ((chunk ^ (r & 7)) << 4)) = make_uint4(outw[0], outw[1], outw[2], outw[3]);
         }
-        fence_proxy_async_smem();
+        // A tile of the stage in tensor memory: lane = row (this warp's quadrant), column = k / 2
+        tmem_st16(tmem_d + ((uint32_t)((warp & 3) * 32) << 16) + kAccCols +
+                      (uint32_t)(s * kATmemColsPerStage + h * 16), outw);
+        tcgen05_fence_before();
         mbar_arrive(bar_deq(s));
       }
       if (!ok) *abort_flag = 1;
     }
     // epilogue: TMEM lane = output feature, column = token
-    if (ok && mbar_wait(bar_acc, 0u, abort_flag)) {
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok && __all_sync(0xffffffffu, mbar_wait(bar_acc, 0u, abort_flag))) {
       tcgen05_fence_after();
       const int quad = warp & 3;                          // TMEM lane quadrant this warp may read
       const int colhalf = (warp - kFirstDeqWarp) >> 2;    // 0 or 1
@@ -500,7 +534,7 @@ int pick_tok_tile(int M) {
 
 template <int TOK, bool DEQUANT, int OUT_MODE>
 int launch_one(const CUtensorMap& tx, const CUtensorMap& tw, const GemmParams& p, dim3 grid, cudaStream_t st) {
-  using Plan = SmemPlan<TOK>;
+  using Plan = SmemPlan<TOK, DEQUANT>;
   auto kern = w4a16_gemm_kernel<TOK, DEQUANT, OUT_MODE>;
   static bool configured = false;           // per instantiation
   if (!configured) {

@@ -1,0 +1,96 @@
+"""Standalone perturbed W4A16 GEMM sweep (K x N and token counts of the paper-shaped linears).
+
+    python -m paper_2505_13430_b200.gemm_sweep [--shapes KxN,...] [--tokens M,...] [--iters I] [--json]
+
+For every shape it times qzo_perturbed_gemm with CUDA events, rotating through enough distinct
+weight / scale / activation sets that every launch streams its operands from HBM (the rotation
+exceeds the L2 capacity), and prints the achieved fraction of the roofline
+max(bytes / HBM bandwidth, flops / dense bf16 peak) with
+bytes = K N / 2 + 2 ceil(K/128) N + 2 M K + 2 M N and flops = 2 M K N.
+"""
+import argparse
+import json
+import os
+
+import torch
+
+from . import inputs, qzo
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+L2_BYTES = 126 * 2 ** 20
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return p["hbm_gbs"], p["bf16_tflops"], "measured"
+    return 6650.0, 1590.0, "fallback"
+
+
+def gemm_bytes(M, K, N):
+    return K * N // 2 + 2 * ((K + 127) // 128) * N + 2 * M * K + 2 * M * N
+
+
+def run_shape(M, K, N, iters, sign=1):
+    per_set = gemm_bytes(M, K, N)
+    n_sets = max(2, min(64, (2 * L2_BYTES) // per_set + 1))
+    sets = []
+    for i in range(n_sets):
+        x = torch.randn((M, K), device="cuda", dtype=torch.float32).bfloat16()
+        words = torch.randint(-2 ** 31, 2 ** 31 - 1, (K // 8, N), device="cuda", dtype=torch.int32)
+        s = (torch.rand(((K + 127) // 128, N), device="cuda") * 0.015 + 0.005).bfloat16()
+        wq = qzo.qzo_repack_int4(words, K, N)
+        y = torch.empty((M, N), device="cuda", dtype=torch.bfloat16)
+        sets.append((x, wq, s, y))
+        del words
+    need = qzo.qzo_gemm_workspace_bytes(M, K, N)
+    ws = torch.empty((max(need, 256),), dtype=torch.uint8, device="cuda")
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+
+    def call(i):
+        x, wq, s, y = sets[i % n_sets]
+        qzo.qzo_perturbed_gemm(x, wq, s, M, K, N, 42, 0, sign, 1e-3, y=y, workspace=ws, status=status)
+
+    for i in range(max(3, n_sets)):
+        call(i)
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for i in range(iters):
+        call(i)
+    ev1.record()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    return ev0.elapsed_time(ev1) * 1e3 / iters, n_sets      # microseconds
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--shapes", default=",".join(f"{k}x{n}" for k, n in inputs.GEMM_SWEEP_KN))
+    ap.add_argument("--tokens", default=",".join(str(m) for m in inputs.GEMM_SWEEP_M))
+    ap.add_argument("--iters", type=int, default=50)
+    ap.add_argument("--json", action="store_true")
+    args = ap.parse_args()
+    bw, tf, src = peaks()
+    rows = []
+    for shape in args.shapes.split(","):
+        K, N = (int(v) for v in shape.split("x"))
+        for M in (int(v) for v in args.tokens.split(",")):
+            us, n_sets = run_shape(M, K, N, args.iters)
+            t_hbm = gemm_bytes(M, K, N) / (bw * 1e9) * 1e6
+            t_mma = 2.0 * M * K * N / (tf * 1e12) * 1e6
+            roof = max(t_hbm, t_mma)
+            rows.append({"K": K, "N": N, "M": M, "us": us, "roofline_us": roof, "bound": "hbm" if t_hbm > t_mma else "tensor",
+                         "frac": roof / us, "tflops": 2.0 * M * K * N / us / 1e6, "gbs": gemm_bytes(M, K, N) / us / 1e3,
+                         "rotation_sets": n_sets})
+            r = rows[-1]
+            if not args.json:
+                print(f"K={K:6d} N={N:6d} M={M:5d}  {us:9.2f} us  roofline {roof:8.2f} us ({r['bound']:6s})  "
+                      f"frac {r['frac']:.3f}  {r['tflops']:8.1f} TFLOP/s  {r['gbs']:8.1f} GB/s  sets={n_sets}", flush=True)
+    if args.json:
+        print(json.dumps({"peaks": {"hbm_gbs": bw, "bf16_tflops": tf, "source": src}, "rows": rows}))
+
+
+if __name__ == "__main__":
+    main()
