@@ -100,7 +100,7 @@ int qzo_gemm_workspace_bytes(int M, int K, int N, size_t* bytes);
  *   i = scale_index_base + (k/128) N + n; the perturbed scale is formed in fp32 inside the
  *   de-quantisation prologue; the stored scales are never modified.
  * d_x bf16 [M][K] row-major; d_wq kernel layout (qzo_repack_int4); d_scales bf16 [G][N];
- * d_bias float [N] or NULL; d_y bf16 [M][N].  sign in {-1, 0, +1} (0 = unperturbed).
+ * d_bias float [N] or NULL; d_y bf16 [M][N], 16-byte aligned.  sign in {-1, 0, +1} (0 = unperturbed).
  * d_workspace: qzo_gemm_workspace_bytes, 256-aligned (may be NULL when that is 0).
  * d_status: int on the device, set non-zero if a bounded wait expired (may be NULL). */
 int qzo_perturbed_gemm(const void* d_x_bf16, const void* d_wq, const void* d_scales_bf16,

@@ -6,23 +6,31 @@
 // written.  The contraction runs on the tcgen05 tensor cores with the accumulator in TMEM.
 //
 // Tile roles.  The de-quantised weight tile is the MMA's A operand (UMMA M = 128 output
-// features), the activation tile is the B operand (UMMA N = TOK tokens, 16..256), so that
-// one de-quantised weight feeds TOK multiply-adds and small token counts do not waste
-// tensor rows.  D[n][t] sits in TMEM with lane = output feature, column = token.
+// features) and lives in tensor memory; the activation tile is the B operand (UMMA N = TOK
+// tokens, 16..256) in shared memory, so that one de-quantised weight feeds TOK multiply-adds
+// and small token counts do not waste tensor rows.  D[n][t] sits in TMEM with lane = output
+// feature, column = token.
 //
-// Warp roles (12 warps):
-//   warp 0      TMA producer: activation tile (2-D tensor map, 128-byte swizzle), packed
-//               int4 tile (one 4 KiB bulk copy), raw bf16 scales of a group (bulk copy)
-//   warp 1      MMA issuer (one elected lane), owns the TMEM allocation
-//   warps 2-3   scale warps: Philox4x32-10 + Box-Muller, s' = s + sign eps z in fp32, split
-//               into bf16 hi + lo parts, written to a small shared-memory ring
-//   warps 4-11  de-quantisers: nibbles -> bf16 (u - 8) * s' into the swizzled K-major
-//               A tile; afterwards the epilogue (TMEM -> registers -> global)
+// The kernel is persistent: one CTA per SM walks a static list of work units (a 128-feature x
+// TOK-token tile of one linear, optionally one K slice of it).  Up to three linears that share
+// the activations (q, k, v or gate, up) are served by one launch; the logical scale index of a
+// scale never depends on that grouping.
+//
+// Warp roles (21 warps):
+//   warp 0       TMA producer of the B ring: activation tiles (2-D tensor map, 128-byte swizzle)
+//   warp 1       MMA issuer (one elected lane), owns the TMEM allocation
+//   warp 2       TMA producer of the A ring: packed int4 tiles (one 4 KiB bulk copy per k-block)
+//   warps 3-4    scale warps: Philox4x32-10 + Box-Muller, s' = s + sign eps z in fp32, split
+//                into bf16 hi + lo parts, written to a small shared-memory ring
+//   warps 5-12   de-quantisers: nibbles -> bf16 (u - 8) * s' written to the A stage in TMEM
+//   warps 13-20  epilogue: TMEM -> registers (+ bias) -> bf16 rows in shared memory -> TMA stores;
+//                runs while the other warps already work on the next unit
 // Every wait on an mbarrier is bounded; when a wait expires the CTA records an error in
 // the status word, drains its copies and leaves through the common exit (TMEM is freed).
 #include "qzo_common.cuh"
 #include "philox.cuh"
 #include "launch.cuh"
+#include "layers.cuh"
 
 #include <cuda.h>
 #include <mutex>
@@ -31,35 +39,43 @@ namespace qzo {
 
 namespace {
 
-constexpr int kStagesDequant = 6;     // pipeline depth over k-blocks, int4 path (A operand lives in TMEM)
-constexpr int kStagesBf16 = 4;        // bf16-weight path (A operand tile in shared memory)
 constexpr int kATmemColsPerStage = kBlockK / 2;   // 64 bf16 along K = 32 TMEM columns of 32 bits
-constexpr int kScaleSlots = 4;        // ring of perturbed-scale rows (one per quantisation group)
-constexpr int kNumScaleWarps = 2;
+constexpr int kScaleSlots = 8;        // ring of perturbed-scale rows (one per quantisation group)
+constexpr int kNumScaleWarps = 4;
 constexpr int kNumDeqWarps = 8;
-constexpr int kFirstScaleWarp = 2;
-constexpr int kFirstDeqWarp = 4;
-constexpr int kNumWarps = kFirstDeqWarp + kNumDeqWarps;
+constexpr int kNumEpiWarps = 8;
+constexpr int kAProducerWarp = 2;
+constexpr int kFirstScaleWarp = 3;
+constexpr int kFirstDeqWarp = kFirstScaleWarp + kNumScaleWarps;
+constexpr int kFirstEpiWarp = kFirstDeqWarp + kNumDeqWarps;
+constexpr int kNumWarps = kFirstEpiWarp + kNumEpiWarps;
 constexpr int kThreads = kNumWarps * 32;
-constexpr int kDeqThreads = kNumDeqWarps * 32;
 constexpr long long kWaitLimitCycles = 4000000000LL;   // ~2 s at boost clock
+constexpr int kSmemBudget = 227 * 1024;
 
-constexpr int kWTileBytes = kTileN * kBlockK * 2;      // 16 KiB bf16 A tile
-constexpr int kRawScaleBytes = kTileN * 2;             // 256 B
+constexpr int kWTileBytes = kTileN * kBlockK * 2;      // 16 KiB bf16 A tile (bf16-weight path)
 constexpr int kCookedScaleBytes = kTileN * 8;          // {hi,hi},{lo,lo} per output feature
 
 enum OutMode { kOutBf16 = 0, kOutF32 = 1 };
 
-struct GemmParams {
+struct LinearDesc {
   const uint8_t* wq;              // kernel-layout int4 (dequant mode)
   const __nv_bfloat16* scales;    // [G][N] of this linear
   const float* bias;              // [N] or null
-  const __nv_bfloat16* residual;  // [M][ldo] or null (added in the epilogue, may alias out)
   void* out;                      // bf16 [M][ldo]  or  float [splits][M][ldo]
-  int M, K, N, ldo;
+  unsigned long long idx_base;    // logical index of scale [0][0]
+  int N, ldo;
+  int n_tiles;                    // ceil(N / 128)
+};
+
+struct GemmParams {
+  LinearDesc lin[kMaxGroupedLinears];
+  int n_lin, tiles_n_total;
+  int M, K;
   int num_kb;                     // ceil(K / 64)
-  int kb_per_split;               // even number of k-blocks per blockIdx.z
-  uint64_t seed, idx_base;
+  int kb_per_split;               // even number of k-blocks per K slice
+  int splits, m_tiles, total_units;
+  unsigned long long seed;
   float sign_eps;                 // sign * eps (0 when unperturbed)
   int* status;
 };
@@ -88,17 +104,56 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// Up to 1024 polls of the barrier in a short loop; true when the phase completed.
+__device__ __forceinline__ bool mbar_poll(uint32_t bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .u32 n;\n\t"
+      "mov.u32 n, 1024;\n"
+      "POLL:\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "@p bra.uni DONE;\n\t"
+      "sub.u32 n, n, 1;\n\t"
+      "setp.ne.u32 p, n, 0;\n\t"
+      "@p bra.uni POLL;\n\t"
+      "mov.u32 %0, 0;\n\t"
+      "bra.uni END;\n"
+      "DONE:\n\t"
+      "mov.u32 %0, 1;\n"
+      "END:\n\t}"
+      : "=r"(done)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return done != 0;
+}
 // Bounded wait: false when the limit expired or another thread of the CTA already gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_poll(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+    if (mbar_poll(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kWaitLimitCycles) return false;
+  }
+}
+// Same bound, for waits that are long and not latency-critical: sleeps between polls so that the
+// waiting warp leaves the issue slots to the working ones.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t i = 1;; ++i) {
+    __nanosleep(256);
     if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 0xFF) == 0) {
+    if ((i & 0x3F) == 0) {
       if (*abort_flag) return false;
       if (clock64() - t0 > kWaitLimitCycles) return false;
     }
   }
+}
+// Hardware barrier among `nthreads` threads of the CTA (whole warps): the waiting warps are parked,
+// they do not poll.  Every participating warp reaches every such barrier, also after a failed wait.
+__device__ __forceinline__ void named_bar_sync(uint32_t id, uint32_t nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
   asm volatile(
@@ -106,6 +161,16 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y)
       : "memory");
 }
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+      ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_group_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_group0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -185,22 +250,71 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16(int m, int n) {
 }
 
 // ----------------------------------------------------------------------------- shared memory plan
-template <int TOK, bool DEQUANT>
+constexpr int cmin(int a, int b) { return a < b ? a : b; }
+
+// Two rings feed the MMA.  The A ring (packed nibbles in shared memory -> de-quantised bf16 in
+// tensor memory) is deep and cheap, so the de-quantisers run well ahead of the tensor pipe; the
+// B ring holds the activation tiles.  A finished bf16 tile leaves in passes of up to 64 tokens
+// through two staging buffers, each pass as one TMA store.
+template <int TOK, bool DEQUANT, int OUT_MODE>
 struct SmemPlan {
-  static constexpr int kStages = DEQUANT ? kStagesDequant : kStagesBf16;
+  static constexpr int kAccCols = TOK < 32 ? 32 : TOK;
   static constexpr int kXTileBytes = TOK * kBlockK * 2;
-  // int4 path: [X tile | packed nibbles]; bf16 path: [W tile | X tile]
-  static constexpr int kStageBytes = DEQUANT ? (kXTileBytes + kPackedTileBytes) : (kWTileBytes + kXTileBytes);
-  static constexpr int kOffW = 0;                                   // bf16 path only
-  static constexpr int kOffX = DEQUANT ? 0 : kWTileBytes;
-  static constexpr int kOffP = kXTileBytes;                         // int4 path only
-  static constexpr int kOffRaw = kStages * kStageBytes;
-  static constexpr int kOffCooked = kOffRaw + kScaleSlots * kRawScaleBytes;
+  // int4 path: A stage = 4 KiB of packed nibbles; bf16 path: A stage = 16 KiB bf16 tile (read by the MMA)
+  static constexpr int kAStageBytes = DEQUANT ? kPackedTileBytes : kWTileBytes;
+  static constexpr int kAStages = DEQUANT ? cmin(6, (512 - kAccCols) / kATmemColsPerStage) : 4;
+  static constexpr int kPassTok = TOK < 64 ? TOK : 64;
+  static constexpr int kPasses = TOK / kPassTok;
+  static constexpr int kStagingBufBytes = kPassTok * kTileN * 2;
+  static constexpr int kStagingBytes = OUT_MODE == kOutBf16 ? 2 * kStagingBufBytes : 0;
+  static constexpr int kFixedBytes = kAStages * kAStageBytes + kStagingBytes + kScaleSlots * kCookedScaleBytes + 1024 + 1024;
+  static constexpr int kBStages = DEQUANT ? cmin(8, (kSmemBudget - kFixedBytes) / kXTileBytes) : kAStages;
+  static_assert(kBStages >= 2 && kAStages >= 2, "pipelines need at least two stages");
+  static constexpr int kOffB = 0;
+  static constexpr int kOffA = kBStages * kXTileBytes;
+  static constexpr int kOffStaging = kOffA + kAStages * kAStageBytes;
+  static constexpr int kOffCooked = kOffStaging + kStagingBytes;
   static constexpr int kOffBars = kOffCooked + kScaleSlots * kCookedScaleBytes;
-  static constexpr int kNumBars = 3 * kStages + 4 * kScaleSlots + 1;
+  static constexpr int kNumBars = 2 * kBStages + 3 * kAStages + 2 * kScaleSlots + 2;
   static constexpr int kOffMisc = kOffBars + kNumBars * 8;
-  static constexpr int kTotal = kOffMisc + 16;
+  static constexpr int kTotal = kOffMisc + 32;
   static constexpr int kDynamicBytes = kTotal + 1024;      // slack for the 1024-byte alignment
+  static_assert(kDynamicBytes <= kSmemBudget, "shared memory budget");
+  static constexpr uint32_t kUsedCols = DEQUANT ? kAccCols + kAStages * kATmemColsPerStage : kAccCols;
+  static constexpr uint32_t kTmemCols = kUsedCols <= 32 ? 32 : kUsedCols <= 64 ? 64 : kUsedCols <= 128 ? 128
+                                        : kUsedCols <= 256 ? 256 : 512;
+  static_assert(kUsedCols <= 512, "TMEM budget");
+};
+
+struct Unit {
+  int lin, n0, tok0, z, kb_begin, nkb;
+};
+// Work unit u of the launch: K slice z, token tile, then the feature tiles of every linear.
+// Consecutive units (which run at the same time on different SMs) share the activation tile.
+__device__ __forceinline__ Unit decode_unit(const GemmParams& p, int u, int tok_tile) {
+  Unit w;
+  const int per = p.tiles_n_total * p.m_tiles;
+  w.z = u / per;
+  const int r = u - w.z * per;
+  const int m = r / p.tiles_n_total;
+  int nn = r - m * p.tiles_n_total;
+  int lin = 0;
+  while (lin + 1 < p.n_lin && nn >= p.lin[lin].n_tiles) { nn -= p.lin[lin].n_tiles; ++lin; }
+  w.lin = lin;
+  w.n0 = nn * kTileN;
+  w.tok0 = m * tok_tile;
+  w.kb_begin = w.z * p.kb_per_split;
+  w.nkb = min(w.kb_begin + p.kb_per_split, p.num_kb) - w.kb_begin;      // >= 1 by construction of the grid
+  return w;
+}
+
+// Ring position: stage index and the parity of the round it is in.
+struct Ring {
+  int s = 0;
+  uint32_t ph = 0;
+  __device__ __forceinline__ void next(int stages) {
+    if (++s == stages) { s = 0; ph ^= 1u; }
+  }
 };
 
 // ----------------------------------------------------------------------------- the kernel
@@ -209,9 +323,13 @@ struct SmemPlan {
 template <int TOK, bool DEQUANT, int OUT_MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
-                  const GemmParams p) {
-  using Plan = SmemPlan<TOK, DEQUANT>;
-  constexpr int kStages = Plan::kStages;
+                  const __grid_constant__ CUtensorMap tmap_y0, const __grid_constant__ CUtensorMap tmap_y1,
+                  const __grid_constant__ CUtensorMap tmap_y2, const __grid_constant__ GemmParams p) {
+  using Plan = SmemPlan<TOK, DEQUANT, OUT_MODE>;
+  constexpr int kAStages = Plan::kAStages;
+  constexpr int kBStages = Plan::kBStages;
+  constexpr uint32_t kAccCols = Plan::kAccCols;
+  constexpr uint32_t kTmemCols = Plan::kTmemCols;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* const smem = smem_raw + (base - smem_u32(smem_raw));
@@ -220,46 +338,43 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
   const int lane = threadIdx.x & 31;
 
   const uint32_t bar0 = base + Plan::kOffBars;
-  auto bar_full = [&](int s) { return bar0 + 8u * s; };                          // TMA landed (X, packed / W)
-  auto bar_deq = [&](int s) { return bar0 + 8u * (kStages + s); };              // A tile de-quantised
-  auto bar_empty = [&](int s) { return bar0 + 8u * (2 * kStages + s); };        // MMAs of the stage retired
-  auto bar_raw_full = [&](int g) { return bar0 + 8u * (3 * kStages + g); };
-  auto bar_raw_empty = [&](int g) { return bar0 + 8u * (3 * kStages + kScaleSlots + g); };
-  auto bar_sc_full = [&](int g) { return bar0 + 8u * (3 * kStages + 2 * kScaleSlots + g); };
-  auto bar_sc_empty = [&](int g) { return bar0 + 8u * (3 * kStages + 3 * kScaleSlots + g); };
-  const uint32_t bar_acc = bar0 + 8u * (3 * kStages + 4 * kScaleSlots);
+  auto bar_b_full = [&](int s) { return bar0 + 8u * s; };                        // activation tile landed
+  auto bar_b_empty = [&](int s) { return bar0 + 8u * (kBStages + s); };          // MMAs that read it retired
+  auto bar_a_full = [&](int s) { return bar0 + 8u * (2 * kBStages + s); };       // packed nibbles / bf16 weights landed
+  auto bar_a_deq = [&](int s) { return bar0 + 8u * (2 * kBStages + kAStages + s); };      // A stage de-quantised
+  auto bar_a_empty = [&](int s) { return bar0 + 8u * (2 * kBStages + 2 * kAStages + s); };  // MMAs that read it retired
+  const uint32_t bar_sc0 = bar0 + 8u * (2 * kBStages + 3 * kAStages);
+  auto bar_sc_full = [&](int g) { return bar_sc0 + 8u * g; };
+  auto bar_sc_empty = [&](int g) { return bar_sc0 + 8u * (kScaleSlots + g); };
+  const uint32_t bar_acc_full = bar_sc0 + 8u * (2 * kScaleSlots);                // accumulator complete
+  const uint32_t bar_acc_empty = bar_acc_full + 8u;                              // accumulator drained
   volatile int* const abort_flag = reinterpret_cast<volatile int*>(smem + Plan::kOffMisc);
   uint32_t* const tmem_slot = reinterpret_cast<uint32_t*>(smem + Plan::kOffMisc + 4);
   volatile int* const never_set = reinterpret_cast<volatile int*>(smem + Plan::kOffMisc + 8);   // stays 0
-
-  const int n0 = blockIdx.x * kTileN;
-  const int tok0 = blockIdx.y * TOK;
-  const int kb_begin = blockIdx.z * p.kb_per_split;
-  const int kb_end = min(kb_begin + p.kb_per_split, p.num_kb);
-  const int nkb = kb_end - kb_begin;                     // >= 1 by construction of the grid
-
-  // TMEM columns: accumulator [0, TOK), then (int4 path) one 32-column A tile per stage
-  constexpr uint32_t kAccCols = TOK < 32 ? 32 : TOK;
-  constexpr uint32_t kUsedCols = DEQUANT ? kAccCols + kStages * kATmemColsPerStage : kAccCols;
-  constexpr uint32_t kTmemCols = kUsedCols <= 32 ? 32 : kUsedCols <= 64 ? 64 : kUsedCols <= 128 ? 128
-                                 : kUsedCols <= 256 ? 256 : 512;
-  static_assert(kUsedCols <= 512, "TMEM budget");
+  // The epilogue warps parked on a hardware barrier learn from this whether their polling warp gave
+  // up: it holds the first unit count that must not be started.  Written by that warp only, before it
+  // reaches the barrier, so that every warp leaves the loop at the same barrier.
+  volatile int* const epi_stop = reinterpret_cast<volatile int*>(smem + Plan::kOffMisc + 12);
 
   if (threadIdx.x == 0) {
     *abort_flag = 0;
     *never_set = 0;
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(bar_full(s), 1);
-      mbar_init(bar_deq(s), kDeqThreads);
-      mbar_init(bar_empty(s), 1);
+    *epi_stop = 0x7fffffff;
+    for (int s = 0; s < kBStages; ++s) {
+      mbar_init(bar_b_full(s), 1);
+      mbar_init(bar_b_empty(s), 1);
+    }
+    for (int s = 0; s < kAStages; ++s) {
+      mbar_init(bar_a_full(s), 1);
+      mbar_init(bar_a_deq(s), kNumDeqWarps);
+      mbar_init(bar_a_empty(s), 1);
     }
     for (int g = 0; g < kScaleSlots; ++g) {
-      mbar_init(bar_raw_full(g), 1);
-      mbar_init(bar_raw_empty(g), 32);
-      mbar_init(bar_sc_full(g), 32);
-      mbar_init(bar_sc_empty(g), kDeqThreads);
+      mbar_init(bar_sc_full(g), 1);
+      mbar_init(bar_sc_empty(g), kNumDeqWarps);
     }
-    mbar_init(bar_acc, 1);
+    mbar_init(bar_acc_full, 1);
+    mbar_init(bar_acc_empty, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
@@ -270,202 +385,261 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
 
   bool ok = true;
 
-  if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+  if (warp == 0 || warp == kAProducerWarp) {
+    // ------------------------------------------------------------------ TMA producers
+    // warp 0 feeds the B ring (activation tiles), warp 2 the A ring (packed nibbles / bf16 weights)
     if (lane == 0) {
+      const bool is_b = warp == 0;
+      const int stages = is_b ? kBStages : kAStages;
+      Ring ring;
       int issued = 0;
-      for (int it = 0; it < nkb; ++it) {
-        const int s = it % kStages;
-        const uint32_t ph = (uint32_t)(it / kStages) & 1u;
-        const int kb = kb_begin + it;
-        if (!mbar_wait(bar_empty(s), ph ^ 1u, abort_flag)) { ok = false; break; }
-        const uint32_t stage = base + s * Plan::kStageBytes;
-        if (DEQUANT) {
-          mbar_arrive_expect_tx(bar_full(s), Plan::kXTileBytes + kPackedTileBytes);
-          bulk_load(stage + Plan::kOffP,
-                    p.wq + ((size_t)blockIdx.x * p.num_kb + kb) * kPackedTileBytes, kPackedTileBytes, bar_full(s));
-        } else {
-          mbar_arrive_expect_tx(bar_full(s), Plan::kXTileBytes + kWTileBytes);
-          tma_load_2d(stage + Plan::kOffW, &tmap_w, bar_full(s), kb * kBlockK, n0);
-        }
-        tma_load_2d(stage + Plan::kOffX, &tmap_x, bar_full(s), kb * kBlockK, tok0);
-        issued = it + 1;
-        if (DEQUANT && ((it & 1) == 0)) {
-          // first k-block of a quantisation group: fetch the group's raw scales
-          const int gi = it >> 1;
-          const int slot = gi % kScaleSlots;
-          const uint32_t gph = (uint32_t)(gi / kScaleSlots) & 1u;
-          if (!mbar_wait(bar_raw_empty(slot), gph ^ 1u, abort_flag)) { ok = false; break; }
-          const int g = (kb >> 1);
-          const int valid = min(kTileN, p.N - n0);
-          const uint32_t bytes = (uint32_t)valid * 2u;
-          mbar_arrive_expect_tx(bar_raw_full(slot), bytes);
-          bulk_load(base + Plan::kOffRaw + slot * kRawScaleBytes, p.scales + (size_t)g * p.N + n0, bytes,
-                    bar_raw_full(slot));
+      for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x) {
+        const Unit w = decode_unit(p, u, TOK);
+        const LinearDesc& L = p.lin[w.lin];
+        for (int it = 0; it < w.nkb; ++it) {
+          const int kb = w.kb_begin + it;
+          if (is_b) {
+            if (!mbar_wait(bar_b_empty(ring.s), ring.ph ^ 1u, abort_flag)) { ok = false; break; }
+            mbar_arrive_expect_tx(bar_b_full(ring.s), Plan::kXTileBytes);
+            tma_load_2d(base + Plan::kOffB + ring.s * Plan::kXTileBytes, &tmap_x, bar_b_full(ring.s), kb * kBlockK, w.tok0);
+          } else {
+            if (!mbar_wait(bar_a_empty(ring.s), ring.ph ^ 1u, abort_flag)) { ok = false; break; }
+            mbar_arrive_expect_tx(bar_a_full(ring.s), Plan::kAStageBytes);
+            const uint32_t dst = base + Plan::kOffA + ring.s * Plan::kAStageBytes;
+            if (DEQUANT)
+              bulk_load(dst, L.wq + ((size_t)(w.n0 / kTileN) * p.num_kb + kb) * kPackedTileBytes, kPackedTileBytes,
+                        bar_a_full(ring.s));
+            else
+              tma_load_2d(dst, &tmap_w, bar_a_full(ring.s), kb * kBlockK, w.n0);
+          }
+          ring.next(stages);
+          ++issued;
         }
       }
       if (!ok) {
         // drain: give the copies already issued a bounded chance to land before the CTA exits
         *abort_flag = 1;
-        for (int it = max(0, issued - kStages); it < issued; ++it)
-          mbar_wait(bar_full(it % kStages), (uint32_t)(it / kStages) & 1u, never_set);
+        const int pending = min(issued, stages);
+        for (int j = 0; j < pending; ++j) {
+          const int idx = issued - 1 - j;
+          const uint32_t bar = is_b ? bar_b_full(idx % stages) : bar_a_full(idx % stages);
+          mbar_wait(bar, (uint32_t)(idx / stages) & 1u, never_set);
+        }
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc = umma_idesc_bf16(kTileN, TOK);
-      for (int it = 0; it < nkb; ++it) {
-        const int s = it % kStages;
-        const uint32_t ph = (uint32_t)(it / kStages) & 1u;
-        if (!mbar_wait(bar_full(s), ph, abort_flag)) { ok = false; break; }
-        if (DEQUANT) {
-          if (!mbar_wait(bar_deq(s), ph, abort_flag)) { ok = false; break; }
-        }
+      Ring ra, rb;
+      int useq = 0;
+      for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x, ++useq) {
+        const Unit w = decode_unit(p, u, TOK);
+        // the epilogue warps must have drained the previous unit's accumulator
+        if (!mbar_wait(bar_acc_empty, ((uint32_t)useq & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         tcgen05_fence_after();
-        const uint32_t stage = base + s * Plan::kStageBytes;
-        const uint64_t bdesc = umma_desc_k_major_sw128(stage + Plan::kOffX);
-        if (DEQUANT) {
-          const uint32_t a_tmem = tmem_d + kAccCols + (uint32_t)(s * kATmemColsPerStage);
+        for (int it = 0; it < w.nkb; ++it) {
+          if (!mbar_wait(DEQUANT ? bar_a_deq(ra.s) : bar_a_full(ra.s), ra.ph, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(bar_b_full(rb.s), rb.ph, abort_flag)) { ok = false; break; }
+          tcgen05_fence_after();
+          const uint64_t bdesc = umma_desc_k_major_sw128(base + Plan::kOffB + rb.s * Plan::kXTileBytes);
+          if (DEQUANT) {
+            const uint32_t a_tmem = tmem_d + kAccCols + (uint32_t)(ra.s * kATmemColsPerStage);
 #pragma unroll
-          for (int k = 0; k < kBlockK / 16; ++k)      // 16 bf16 along K = 8 TMEM columns
-            umma_bf16_tmem_a(tmem_d, a_tmem + (uint32_t)(k * 8), bdesc + (uint64_t)(k * 2), idesc,
-                             (it > 0 || k > 0) ? 1u : 0u);
-        } else {
-          const uint64_t adesc = umma_desc_k_major_sw128(stage + Plan::kOffW);
+            for (int k = 0; k < kBlockK / 16; ++k)      // 16 bf16 along K = 8 TMEM columns
+              umma_bf16_tmem_a(tmem_d, a_tmem + (uint32_t)(k * 8), bdesc + (uint64_t)(k * 2), idesc,
+                               (it > 0 || k > 0) ? 1u : 0u);
+          } else {
+            const uint64_t adesc = umma_desc_k_major_sw128(base + Plan::kOffA + ra.s * Plan::kAStageBytes);
 #pragma unroll
-          for (int k = 0; k < kBlockK / 16; ++k)
-            umma_bf16(tmem_d, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
-                      (it > 0 || k > 0) ? 1u : 0u);
+            for (int k = 0; k < kBlockK / 16; ++k)
+              umma_bf16(tmem_d, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
+                        (it > 0 || k > 0) ? 1u : 0u);
+          }
+          umma_commit(bar_a_empty(ra.s));
+          umma_commit(bar_b_empty(rb.s));
+          ra.next(kAStages);
+          rb.next(kBStages);
         }
-        umma_commit(bar_empty(s));
+        if (ok) umma_commit(bar_acc_full);
       }
-      if (ok) umma_commit(bar_acc);
-      else *abort_flag = 1;
+      if (!ok) *abort_flag = 1;
     }
   } else if (warp < kFirstDeqWarp) {
     // ------------------------------------------------------------------ scale warps
     if (DEQUANT) {
       const int sw = warp - kFirstScaleWarp;
-      const int ngroups = (nkb + 1) >> 1;
-      for (int gi = sw; gi < ngroups; gi += kNumScaleWarps) {
-        const int slot = gi % kScaleSlots;
-        const uint32_t gph = (uint32_t)(gi / kScaleSlots) & 1u;
-        const int g = (kb_begin >> 1) + gi;
-        if (!mbar_wait(bar_raw_full(slot), gph, abort_flag)) { ok = false; break; }
-        const __nv_bfloat16* raw = reinterpret_cast<const __nv_bfloat16*>(smem + Plan::kOffRaw + slot * kRawScaleBytes);
-        const int r0 = lane * 4;                       // four consecutive output features = one counter block
-        float sv[4];
+      int gig = 0;                        // quantisation groups visited by this CTA so far (all units)
+      for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x) {
+        const Unit w = decode_unit(p, u, TOK);
+        const LinearDesc& L = p.lin[w.lin];
+        const int ngroups = (w.nkb + 1) >> 1;
+        for (int gi = 0; gi < ngroups; ++gi, ++gig) {
+          if ((gig % kNumScaleWarps) != sw) continue;
+          const int slot = gig % kScaleSlots;
+          const uint32_t gph = (uint32_t)(gig / kScaleSlots) & 1u;
+          const int g = (w.kb_begin >> 1) + gi;
+          const int r0 = lane * 4;                       // four consecutive output features = one counter block
+          float sv[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+          if (w.n0 + r0 < L.N) {                         // N is a multiple of 8: all four or none
+            const uint2 raw = *reinterpret_cast<const uint2*>(L.scales + (size_t)g * L.N + w.n0 + r0);
+            const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
+            const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
+            sv[0] = __low2float(a); sv[1] = __high2float(a); sv[2] = __low2float(b); sv[3] = __high2float(b);
+            if (p.sign_eps != 0.0f) {
+              float z[4];
+              const uint64_t i0 = L.idx_base + (uint64_t)g * (uint64_t)L.N + (uint64_t)(w.n0 + r0);
+              normals_of_block(p.seed, i0 >> 2, z);
 #pragma unroll
-        for (int l = 0; l < 4; ++l) sv[l] = (n0 + r0 + l < p.N) ? __bfloat162float(raw[r0 + l]) : 0.0f;
-        mbar_arrive(bar_raw_empty(slot));
-        if (p.sign_eps != 0.0f) {
-          float z[4];
-          const uint64_t i0 = p.idx_base + (uint64_t)g * (uint64_t)p.N + (uint64_t)(n0 + r0);
-          normals_of_block(p.seed, i0 >> 2, z);
+              for (int l = 0; l < 4; ++l) sv[l] = fmaf(p.sign_eps, z[l], sv[l]);
+            }
+          }
+          uint32_t cooked[8];
 #pragma unroll
-          for (int l = 0; l < 4; ++l) sv[l] = (n0 + r0 + l < p.N) ? fmaf(p.sign_eps, z[l], sv[l]) : 0.0f;
+          for (int l = 0; l < 4; ++l) {
+            const __nv_bfloat16 hi = __float2bfloat16_rn(sv[l]);
+            const __nv_bfloat16 lo = __float2bfloat16_rn(sv[l] - __bfloat162float(hi));
+            const uint32_t h16 = (uint32_t)__bfloat16_as_ushort(hi), l16 = (uint32_t)__bfloat16_as_ushort(lo);
+            cooked[2 * l] = h16 | (h16 << 16);
+            cooked[2 * l + 1] = l16 | (l16 << 16);
+          }
+          if (!__all_sync(0xffffffffu, mbar_wait_relaxed(bar_sc_empty(slot), gph ^ 1u, abort_flag))) { ok = false; break; }
+          uint4* dst = reinterpret_cast<uint4*>(smem + Plan::kOffCooked + slot * kCookedScaleBytes + r0 * 8);
+          dst[0] = make_uint4(cooked[0], cooked[1], cooked[2], cooked[3]);
+          dst[1] = make_uint4(cooked[4], cooked[5], cooked[6], cooked[7]);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_sc_full(slot));
         }
-        uint32_t cooked[8];
-#pragma unroll
-        for (int l = 0; l < 4; ++l) {
-          const __nv_bfloat16 hi = __float2bfloat16_rn(sv[l]);
-          const __nv_bfloat16 lo = __float2bfloat16_rn(sv[l] - __bfloat162float(hi));
-          const uint32_t h16 = (uint32_t)__bfloat16_as_ushort(hi), l16 = (uint32_t)__bfloat16_as_ushort(lo);
-          cooked[2 * l] = h16 | (h16 << 16);
-          cooked[2 * l + 1] = l16 | (l16 << 16);
-        }
-        if (!mbar_wait(bar_sc_empty(slot), gph ^ 1u, abort_flag)) { ok = false; break; }
-        uint4* dst = reinterpret_cast<uint4*>(smem + Plan::kOffCooked + slot * kCookedScaleBytes + r0 * 8);
-        dst[0] = make_uint4(cooked[0], cooked[1], cooked[2], cooked[3]);
-        dst[1] = make_uint4(cooked[4], cooked[5], cooked[6], cooked[7]);
-        mbar_arrive(bar_sc_full(slot));
       }
       if (!ok) *abort_flag = 1;
     }
-  } else {
-    // ------------------------------------------------------------------ de-quantisers, then epilogue
-    const int dt = threadIdx.x - kFirstDeqWarp * 32;      // 0..255
+  } else if (warp < kFirstEpiWarp) {
+    // ------------------------------------------------------------------ de-quantisers
     if (DEQUANT) {
-      const int r = (warp & 3) * 32 + lane;               // row of the tile = TMEM lane this warp may access
-      const int h = dt >> 7;                              // half of the k-block (32 k each)
+      const int dt = threadIdx.x - kFirstDeqWarp * 32;      // 0..255
+      const int r = (warp & 3) * 32 + lane;                 // row of the tile = TMEM lane this warp may access
+      const int h = dt >> 7;                                // half of the k-block (32 k each)
       const __nv_bfloat162 magic_bias = __halves2bfloat162(__float2bfloat16_rn(136.0f), __float2bfloat16_rn(136.0f));
       __nv_bfloat162 s_hi, s_lo;
       *reinterpret_cast<uint32_t*>(&s_hi) = 0u;
       *reinterpret_cast<uint32_t*>(&s_lo) = 0u;
-      for (int it = 0; it < nkb && ok; ++it) {
-        const int s = it % kStages;
-        const uint32_t ph = (uint32_t)(it / kStages) & 1u;
-        if ((it & 1) == 0) {
-          const int gi = it >> 1;
-          const int slot = gi % kScaleSlots;
-          const uint32_t gph = (uint32_t)(gi / kScaleSlots) & 1u;
-          if (!__all_sync(0xffffffffu, mbar_wait(bar_sc_full(slot), gph, abort_flag))) { ok = false; break; }
-          const uint2 c = *reinterpret_cast<const uint2*>(smem + Plan::kOffCooked + slot * kCookedScaleBytes + r * 8);
-          *reinterpret_cast<uint32_t*>(&s_hi) = c.x;
-          *reinterpret_cast<uint32_t*>(&s_lo) = c.y;
-          mbar_arrive(bar_sc_empty(slot));
-        }
-        // bar_full(s) completing implies the stage was released by the MMAs that last read it
-        if (!__all_sync(0xffffffffu, mbar_wait(bar_full(s), ph, abort_flag))) { ok = false; break; }
-        tcgen05_fence_after();                              // orders the MMAs' reads of this A stage before the store below
-        uint8_t* stage = smem + s * Plan::kStageBytes;
-        const uint4 pk = *reinterpret_cast<const uint4*>(stage + Plan::kOffP + (h * kTileN + r) * 16);
-        const uint32_t words[4] = {pk.x, pk.y, pk.z, pk.w};
-        uint32_t outw[16];                                  // k = 32 h + 2 j, 2 j + 1 in register j
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-#pragma unroll
-          for (int pp = 0; pp < 4; ++pp) {
-            uint32_t x = ((words[i] >> (4 * pp)) & 0x000F000Fu) | 0x43004300u;     // bf16x2 {128 + u_lo, 128 + u_hi}
-            __nv_bfloat162 q2 = __hsub2(*reinterpret_cast<__nv_bfloat162*>(&x), magic_bias);   // exact u - 8
-            __nv_bfloat162 w2 = __hfma2(q2, s_hi, __hmul2(q2, s_lo));
-            outw[i * 4 + pp] = *reinterpret_cast<uint32_t*>(&w2);
+      Ring ra;
+      int gig = 0;
+      for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x) {
+        const Unit w = decode_unit(p, u, TOK);
+        for (int it = 0; it < w.nkb; ++it) {
+          if ((it & 1) == 0) {
+            const int slot = gig % kScaleSlots;
+            const uint32_t gph = (uint32_t)(gig / kScaleSlots) & 1u;
+            ++gig;
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_sc_full(slot), gph, abort_flag))) { ok = false; break; }
+            const uint2 c = *reinterpret_cast<const uint2*>(smem + Plan::kOffCooked + slot * kCookedScaleBytes + r * 8);
+            *reinterpret_cast<uint32_t*>(&s_hi) = c.x;
+            *reinterpret_cast<uint32_t*>(&s_lo) = c.y;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_sc_empty(slot));
           }
+          // bar_a_full completing implies the stage was released by the MMAs that last read it
+          if (!__all_sync(0xffffffffu, mbar_wait(bar_a_full(ra.s), ra.ph, abort_flag))) { ok = false; break; }
+          tcgen05_fence_after();                              // orders the MMAs' reads of this A stage before the store below
+          const uint8_t* stage = smem + Plan::kOffA + ra.s * Plan::kAStageBytes;
+          const uint4 pk = *reinterpret_cast<const uint4*>(stage + (h * kTileN + r) * 16);
+          const uint32_t words[4] = {pk.x, pk.y, pk.z, pk.w};
+          uint32_t outw[16];                                  // k = 32 h + 2 j, 2 j + 1 in register j
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+#pragma unroll
+            for (int pp = 0; pp < 4; ++pp) {
+              uint32_t x = ((words[i] >> (4 * pp)) & 0x000F000Fu) | 0x43004300u;     // bf16x2 {128 + u_lo, 128 + u_hi}
+              __nv_bfloat162 q2 = __hsub2(*reinterpret_cast<__nv_bfloat162*>(&x), magic_bias);   // exact u - 8
+              __nv_bfloat162 w2 = __hfma2(q2, s_hi, __hmul2(q2, s_lo));
+              outw[i * 4 + pp] = *reinterpret_cast<uint32_t*>(&w2);
+            }
+          }
+          // A tile of the stage in tensor memory: lane = row (this warp's quadrant), column = k / 2
+          tmem_st16(tmem_d + ((uint32_t)((warp & 3) * 32) << 16) + kAccCols +
+                        (uint32_t)(ra.s * kATmemColsPerStage + h * 16), outw);
+          tcgen05_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_a_deq(ra.s));
+          ra.next(kAStages);
         }
-        // A tile of the stage in tensor memory: lane = row (this warp's quadrant), column = k / 2
-        tmem_st16(tmem_d + ((uint32_t)((warp & 3) * 32) << 16) + kAccCols +
-                      (uint32_t)(s * kATmemColsPerStage + h * 16), outw);
-        tcgen05_fence_before();
-        mbar_arrive(bar_deq(s));
       }
       if (!ok) *abort_flag = 1;
     }
-    // epilogue: TMEM lane = output feature, column = token
-    ok = __all_sync(0xffffffffu, ok);
-    if (ok && __all_sync(0xffffffffu, mbar_wait(bar_acc, 0u, abort_flag))) {
+  } else {
+    // ------------------------------------------------------------------ epilogue
+    // TMEM lane = output feature, column = token.  Only the first epilogue warp polls the mbarrier;
+    // the others are parked on a hardware barrier, which every epilogue warp reaches every time.
+    const int ew = warp - kFirstEpiWarp;
+    const int quad = warp & 3;                          // TMEM lane quadrant this warp may read
+    const int colpart = ew >> 2;                        // 0 or 1: which 16-column chunks this warp takes
+    const int f = quad * 32 + lane;                     // feature within the tile
+    const bool elected = (ew == 0 && lane == 0);
+    constexpr int kChunksPerPass = Plan::kPassTok / 16;
+    int useq = 0;
+    uint32_t passes_done = 0;                           // staging buffer = passes_done & 1
+    bool store_pending = false;
+    for (int u = blockIdx.x; u < p.total_units; u += gridDim.x, ++useq) {
+      const Unit w = decode_unit(p, u, TOK);
+      const LinearDesc& L = p.lin[w.lin];
+      const CUtensorMap* tmap_y = w.lin == 0 ? &tmap_y0 : (w.lin == 1 ? &tmap_y1 : &tmap_y2);
+      const int n = w.n0 + f;
+      const float bias = (L.bias != nullptr && n < L.N && w.z == 0) ? L.bias[n] : 0.0f;
+      if (ew == 0 && !mbar_wait(bar_acc_full, (uint32_t)useq & 1u, abort_flag)) {
+        *epi_stop = useq;
+        __threadfence_block();
+      }
+      named_bar_sync(1, kNumEpiWarps * 32);
+      if (useq >= *epi_stop) { ok = false; break; }
       tcgen05_fence_after();
-      const int quad = warp & 3;                          // TMEM lane quadrant this warp may read
-      const int colhalf = (warp - kFirstDeqWarp) >> 2;    // 0 or 1
-      const int n = n0 + quad * 32 + lane;
-      const float bias = (p.bias != nullptr && n < p.N && blockIdx.z == 0) ? p.bias[n] : 0.0f;
-      constexpr int kChunks = TOK / 16;
-      for (int c = colhalf; c < kChunks; c += 2) {
-        if (tok0 + c * 16 >= p.M) break;                  // warp-uniform
-        uint32_t v[16];
-        tmem_ld16(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)(c * 16), v);
-        if (n < p.N) {
+      if (OUT_MODE == kOutBf16) {
+        for (int pass = 0; pass < Plan::kPasses; ++pass, ++passes_done) {
+          const int tok_pass = w.tok0 + pass * Plan::kPassTok;
+          if (tok_pass >= p.M) break;                       // uniform over the epilogue warps
+          __nv_bfloat16* const buf = reinterpret_cast<__nv_bfloat16*>(smem + Plan::kOffStaging +
+                                                                       (passes_done & 1u) * Plan::kStagingBufBytes);
+          for (int c = colpart; c < kChunksPerPass; c += 2) {
+            uint32_t v[16];
+            tmem_ld16(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)(pass * Plan::kPassTok + c * 16), v);
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const int t = tok0 + c * 16 + j;
-            if (t < p.M) {
-              float acc = __uint_as_float(v[j]) + bias;
-              if (OUT_MODE == kOutF32) {
-                float* o = reinterpret_cast<float*>(p.out) + ((size_t)blockIdx.z * p.M + t) * p.ldo + n;
-                *o = acc;
-              } else {
-                const size_t off = (size_t)t * p.ldo + n;
-                if (p.residual) acc += __bfloat162float(p.residual[off]);
-                reinterpret_cast<__nv_bfloat16*>(p.out)[off] = __float2bfloat16_rn(acc);
-              }
+            for (int j = 0; j < 16; ++j)
+              buf[(c * 16 + j) * kTileN + f] = __float2bfloat16_rn(__uint_as_float(v[j]) + bias);
+          }
+          fence_proxy_async_smem();                         // staged rows visible to the TMA store
+          // the store of the previous pass has read the other buffer, which the next pass will fill
+          if (elected && store_pending) bulk_wait_group_read0();
+          if (pass == Plan::kPasses - 1 || tok_pass + Plan::kPassTok >= p.M) tcgen05_fence_before();
+          named_bar_sync(1, kNumEpiWarps * 32);
+          if (elected) {
+            tma_store_2d(tmap_y, smem_u32(buf), w.n0, tok_pass);
+            bulk_commit_group();
+            store_pending = true;
+          }
+        }
+      } else {
+        constexpr int kChunks = TOK / 16;
+        for (int c = colpart; c < kChunks; c += 2) {
+          if (w.tok0 + c * 16 >= p.M) break;                // warp-uniform
+          uint32_t v[16];
+          tmem_ld16(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)(c * 16), v);
+          if (n < L.N) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int t = w.tok0 + c * 16 + j;
+              if (t < p.M)
+                reinterpret_cast<float*>(L.out)[((size_t)w.z * p.M + t) * L.ldo + n] = __uint_as_float(v[j]) + bias;
             }
           }
         }
+        tcgen05_fence_before();
+        named_bar_sync(1, kNumEpiWarps * 32);
       }
-    } else {
-      ok = false;
-      *abort_flag = 1;
+      // accumulator drained: the MMA warp may start the next unit
+      if (elected) mbar_arrive(bar_acc_empty);
     }
+    if (elected && store_pending) bulk_wait_group0();
+    if (!ok) *abort_flag = 1;
   }
 
   if (!ok && p.status != nullptr) atomicExch(p.status, 1);
@@ -477,19 +651,16 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
   }
 }
 
-// Sum of split-K partials in a fixed order, + bias + residual, to bf16.
+// Sum of split-K partials in a fixed order, + bias, to bf16.
 __global__ void splitk_reduce_kernel(const float* __restrict__ part, int splits, int M, int N,
-                                     const float* __restrict__ bias, const __nv_bfloat16* __restrict__ residual,
-                                     __nv_bfloat16* __restrict__ out, int ldo) {
+                                     const float* __restrict__ bias, __nv_bfloat16* __restrict__ out, int ldo) {
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (int64_t)M * N) return;
   const int t = (int)(idx / N), n = (int)(idx % N);
   float acc = 0.0f;
   for (int z = 0; z < splits; ++z) acc += part[((size_t)z * M + t) * N + n];
   if (bias) acc += bias[n];
-  const size_t off = (size_t)t * ldo + n;
-  if (residual) acc += __bfloat162float(residual[off]);
-  out[off] = __float2bfloat16_rn(acc);
+  out[(size_t)t * ldo + n] = __float2bfloat16_rn(acc);
 }
 
 // ----------------------------------------------------------------------------- host side
@@ -510,17 +681,20 @@ EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
-// 2-D bf16 row-major [rows][cols] tensor map, box = 64 columns x box_rows rows, 128-byte swizzle.
-int make_tmap_bf16(CUtensorMap* map, const void* ptr, int rows, int cols, int box_rows) {
+// 2-D bf16 tensor map of a row-major [rows][ld] matrix of which `cols` columns are addressed;
+// box = box_cols x box_rows.  Operand tiles use the 128-byte swizzle (box_cols = 64); output
+// tiles are plain rows of 128 features.
+int make_tmap_bf16(CUtensorMap* map, const void* ptr, int rows, int cols, int ld, int box_cols, int box_rows,
+                   bool swizzle128) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return QZO_ERR_CUDA;
   cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  cuuint64_t gstride[1] = {(cuuint64_t)cols * 2};
-  cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)box_rows};
+  cuuint64_t gstride[1] = {(cuuint64_t)ld * 2};
+  cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim, gstride, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? QZO_OK : QZO_ERR_CUDA;
 }
 
@@ -532,27 +706,41 @@ int pick_tok_tile(int M) {
   return 256;
 }
 
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+      n = 0;
+    if (n <= 0) n = 148;
+  }
+  return n;
+}
+
 template <int TOK, bool DEQUANT, int OUT_MODE>
-int launch_one(const CUtensorMap& tx, const CUtensorMap& tw, const GemmParams& p, dim3 grid, cudaStream_t st) {
-  using Plan = SmemPlan<TOK, DEQUANT>;
+int launch_one(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorMap* ty, const GemmParams& p,
+               cudaStream_t st) {
+  using Plan = SmemPlan<TOK, DEQUANT, OUT_MODE>;
   auto kern = w4a16_gemm_kernel<TOK, DEQUANT, OUT_MODE>;
   static bool configured = false;           // per instantiation
   if (!configured) {
     QZO_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Plan::kDynamicBytes));
     configured = true;
   }
-  QZO_LAUNCH(kern, grid, dim3(kThreads), Plan::kDynamicBytes, st, tx, tw, p);
+  const int grid = p.total_units < sm_count() ? p.total_units : sm_count();
+  QZO_LAUNCH(kern, dim3(grid), dim3(kThreads), Plan::kDynamicBytes, st, tx, tw, ty[0], ty[1], ty[2], p);
   return QZO_OK;
 }
 
 template <bool DEQUANT, int OUT_MODE>
-int launch_tok(int tok, const CUtensorMap& tx, const CUtensorMap& tw, const GemmParams& p, dim3 grid, cudaStream_t st) {
+int launch_tok(int tok, const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorMap* ty, const GemmParams& p,
+               cudaStream_t st) {
   switch (tok) {
-    case 16: return launch_one<16, DEQUANT, OUT_MODE>(tx, tw, p, grid, st);
-    case 32: return launch_one<32, DEQUANT, OUT_MODE>(tx, tw, p, grid, st);
-    case 64: return launch_one<64, DEQUANT, OUT_MODE>(tx, tw, p, grid, st);
-    case 128: return launch_one<128, DEQUANT, OUT_MODE>(tx, tw, p, grid, st);
-    default: return launch_one<256, DEQUANT, OUT_MODE>(tx, tw, p, grid, st);
+    case 16: return launch_one<16, DEQUANT, OUT_MODE>(tx, tw, ty, p, st);
+    case 32: return launch_one<32, DEQUANT, OUT_MODE>(tx, tw, ty, p, st);
+    case 64: return launch_one<64, DEQUANT, OUT_MODE>(tx, tw, ty, p, st);
+    case 128: return launch_one<128, DEQUANT, OUT_MODE>(tx, tw, ty, p, st);
+    default: return launch_one<256, DEQUANT, OUT_MODE>(tx, tw, ty, p, st);
   }
 }
 
@@ -565,7 +753,7 @@ int gemm_splits(int M, int K, int N) {
   const int tiles = ceil_div(N, kTileN) * ceil_div(M, tok);
   const int groups = ceil_div(K, kGroup);
   if (tiles >= 120 || groups < 8) return 1;
-  int splits = 296 / tiles;                      // aim at two CTAs per SM
+  int splits = 296 / tiles;                      // aim at two units per SM
   if (splits > groups / 4) splits = groups / 4;  // at least four groups per slice
   if (splits > 16) splits = 16;
   return splits < 1 ? 1 : splits;
@@ -577,42 +765,74 @@ size_t gemm_workspace_bytes(int M, int K, int N) {
   return (size_t)splits * M * N * sizeof(float);
 }
 
-// Y = X W' (+ bias) (+ residual) with W' de-quantised from int4 and perturbed scales.
-int launch_perturbed_gemm(const __nv_bfloat16* d_x, const void* d_wq, const __nv_bfloat16* d_scales,
-                          const float* d_bias, const __nv_bfloat16* d_residual, __nv_bfloat16* d_y, int ldo,
-                          int M, int K, int N, uint64_t seed, uint64_t idx_base, int sign, float eps,
-                          void* d_ws, size_t ws_bytes, int* d_status, cudaStream_t st) {
-  if (M <= 0 || K <= 0 || N <= 0 || (K % 8) != 0 || (N % 8) != 0 || (idx_base % 4) != 0) return QZO_ERR_BAD_ARG;
+// Y_j = X W'_j (+ bias_j) for up to three linears that share X, with W'_j de-quantised
+// from int4 and perturbed scales.
+int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const GemmLinear* lins, int n_lin,
+                                uint64_t seed, int sign, float eps, void* d_ws, size_t ws_bytes, int* d_status,
+                                cudaStream_t st) {
+  if (M <= 0 || K <= 0 || (K % 8) != 0 || n_lin < 1 || n_lin > kMaxGroupedLinears) return QZO_ERR_BAD_ARG;
+  for (int j = 0; j < n_lin; ++j)
+    if (lins[j].N <= 0 || (lins[j].N % 8) != 0 || (lins[j].idx_base % 4) != 0 || (lins[j].ldo % 8) != 0)
+      return QZO_ERR_BAD_ARG;
   const int tok = pick_tok_tile(M);
-  CUtensorMap tx;
-  QZO_TRY(make_tmap_bf16(&tx, d_x, M, K, tok));
-  const int splits = gemm_splits(M, K, N);
+  // split-K only pays for small token counts; grouped launches of such problems go one by one
+  if (n_lin > 1) {
+    bool any_split = false;
+    for (int j = 0; j < n_lin; ++j) any_split = any_split || gemm_splits(M, K, lins[j].N) > 1;
+    if (any_split) {
+      for (int j = 0; j < n_lin; ++j)
+        QZO_TRY(launch_perturbed_gemm_group(d_x, M, K, lins + j, 1, seed, sign, eps, d_ws, ws_bytes, d_status, st));
+      return QZO_OK;
+    }
+  }
+  CUtensorMap tx, ty[kMaxGroupedLinears];
+  QZO_TRY(make_tmap_bf16(&tx, d_x, M, K, K, kBlockK, tok, true));
   GemmParams p{};
-  p.wq = reinterpret_cast<const uint8_t*>(d_wq);
-  p.scales = d_scales;
-  p.M = M; p.K = K; p.N = N;
+  p.n_lin = n_lin;
+  p.M = M; p.K = K;
   p.num_kb = ceil_div(K, kBlockK);
-  p.seed = seed; p.idx_base = idx_base;
+  p.m_tiles = ceil_div(M, tok);
+  p.seed = seed;
   p.sign_eps = (float)sign * eps;
   p.status = d_status;
-  const int groups = ceil_div(K, kGroup);
-  if (splits <= 1) {
-    p.bias = d_bias; p.residual = d_residual; p.out = d_y; p.ldo = ldo;
-    p.kb_per_split = ceil_div(p.num_kb, 2) * 2;
-    dim3 grid(ceil_div(N, kTileN), ceil_div(M, tok), 1);
-    return launch_tok<true, kOutBf16>(tok, tx, tx, p, grid, st);
+  const int splits = (n_lin == 1) ? gemm_splits(M, K, lins[0].N) : 1;
+  for (int j = 0; j < n_lin; ++j) {
+    LinearDesc& L = p.lin[j];
+    L.wq = reinterpret_cast<const uint8_t*>(lins[j].wq);
+    L.scales = lins[j].scales;
+    L.idx_base = lins[j].idx_base;
+    L.N = lins[j].N;
+    L.n_tiles = ceil_div(lins[j].N, kTileN);
+    p.tiles_n_total += L.n_tiles;
+    if (splits <= 1) {
+      L.bias = lins[j].bias; L.out = lins[j].out; L.ldo = lins[j].ldo;
+    }
   }
-  const size_t need = (size_t)splits * M * N * sizeof(float);
+  if (splits <= 1) {
+    for (int j = 0; j < kMaxGroupedLinears; ++j) {
+      const GemmLinear& g = lins[j < n_lin ? j : 0];
+      QZO_TRY(make_tmap_bf16(&ty[j], g.out, M, g.N, g.ldo, kTileN, tok < 64 ? tok : 64, false));
+    }
+    p.splits = 1;
+    p.kb_per_split = ceil_div(p.num_kb, 2) * 2;
+    p.total_units = p.tiles_n_total * p.m_tiles;
+    return launch_tok<true, kOutBf16>(tok, tx, tx, ty, p, st);
+  }
+  const GemmLinear& g = lins[0];
+  const int groups = ceil_div(K, kGroup);
+  const size_t need = (size_t)splits * M * g.N * sizeof(float);
   if (d_ws == nullptr || ws_bytes < need) return QZO_ERR_WORKSPACE;
   const int groups_per = ceil_div(groups, splits);
   const int zdim = ceil_div(groups, groups_per);           // every slice is non-empty
-  p.bias = nullptr; p.residual = nullptr; p.out = d_ws; p.ldo = N;
+  p.lin[0].bias = nullptr; p.lin[0].out = d_ws; p.lin[0].ldo = g.N;
+  p.splits = zdim;
   p.kb_per_split = groups_per * 2;
-  dim3 grid(ceil_div(N, kTileN), ceil_div(M, tok), zdim);
-  QZO_TRY((launch_tok<true, kOutF32>(tok, tx, tx, p, grid, st)));
-  const int64_t total = (int64_t)M * N;
+  p.total_units = p.tiles_n_total * p.m_tiles * zdim;
+  ty[0] = ty[1] = ty[2] = tx;                              // unused by the fp32 epilogue
+  QZO_TRY((launch_tok<true, kOutF32>(tok, tx, tx, ty, p, st)));
+  const int64_t total = (int64_t)M * g.N;
   QZO_LAUNCH(splitk_reduce_kernel, dim3((unsigned)ceil_div64(total, 256)), dim3(256), 0, st,
-             reinterpret_cast<const float*>(d_ws), zdim, M, N, d_bias, d_residual, d_y, ldo);
+             reinterpret_cast<const float*>(d_ws), zdim, M, g.N, g.bias, g.out, g.ldo);
   return QZO_OK;
 }
 
@@ -621,17 +841,22 @@ int launch_bf16_gemm_f32out(const __nv_bfloat16* d_x, const __nv_bfloat16* d_w, 
                             int* d_status, cudaStream_t st) {
   if (M <= 0 || K <= 0 || N <= 0 || (K % 8) != 0) return QZO_ERR_BAD_ARG;
   const int tok = pick_tok_tile(M);
-  CUtensorMap tx, tw;
-  QZO_TRY(make_tmap_bf16(&tx, d_x, M, K, tok));
-  QZO_TRY(make_tmap_bf16(&tw, d_w, N, K, kTileN));
+  CUtensorMap tx, tw, ty[kMaxGroupedLinears];
+  QZO_TRY(make_tmap_bf16(&tx, d_x, M, K, K, kBlockK, tok, true));
+  QZO_TRY(make_tmap_bf16(&tw, d_w, N, K, K, kBlockK, kTileN, true));
+  ty[0] = ty[1] = ty[2] = tx;                              // unused by the fp32 epilogue
   GemmParams p{};
-  p.M = M; p.K = K; p.N = N; p.ldo = N;
-  p.out = d_out;
+  p.n_lin = 1;
+  p.lin[0].N = N; p.lin[0].ldo = N; p.lin[0].out = d_out; p.lin[0].n_tiles = ceil_div(N, kTileN);
+  p.tiles_n_total = p.lin[0].n_tiles;
+  p.M = M; p.K = K;
   p.num_kb = ceil_div(K, kBlockK);
   p.kb_per_split = ceil_div(p.num_kb, 2) * 2;
+  p.splits = 1;
+  p.m_tiles = ceil_div(M, tok);
+  p.total_units = p.tiles_n_total * p.m_tiles;
   p.status = d_status;
-  dim3 grid(ceil_div(N, kTileN), ceil_div(M, tok), 1);
-  return launch_tok<false, kOutF32>(tok, tx, tw, p, grid, st);
+  return launch_tok<false, kOutF32>(tok, tx, tw, ty, p, st);
 }
 
 }  // namespace qzo

@@ -61,39 +61,89 @@ __global__ void embedding_kernel(const int32_t* __restrict__ tokens, const __nv_
   }
 }
 
-// y = x * rsqrt(mean(x^2) + eps) * w
-__global__ void rmsnorm_kernel(const __nv_bfloat16* __restrict__ x, const float* __restrict__ w, float eps, int d,
-                               __nv_bfloat16* __restrict__ y) {
-  __shared__ float red[32];
-  const __nv_bfloat16* row = x + (size_t)blockIdx.x * d;
-  float ss = 0.0f;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    const float v = __bfloat162float(row[i]);
-    ss += v * v;
-  }
-  ss = block_sum(ss, red);
-  const float r = rsqrtf(ss / (float)d + eps);
-  __nv_bfloat16* out = y + (size_t)blockIdx.x * d;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) out[i] = __float2bfloat16_rn(__bfloat162float(row[i]) * r * w[i]);
-}
+// Row-wise norms, optionally fused with the residual add that precedes them:
+//   if delta != null:  x <- bf16(x + delta)   (the residual stream, updated in place)
+//   RMSNorm:   y = x * rsqrt(mean(x^2) + eps) * w
+//   LayerNorm: y = (x - mean) * rsqrt(var + eps) * w + b
+// One CTA per row; the row lives in registers between the statistics and the output (16-byte
+// accesses, d a multiple of 8, up to kNormVecs * 256 * 8 elements per row).  y may alias delta.
+constexpr int kNormThreads = 256;
+constexpr int kNormVecs = 4;
 
-// y = (x - mean) * rsqrt(var + eps) * w + b
-__global__ void layernorm_kernel(const __nv_bfloat16* __restrict__ x, const float* __restrict__ w,
-                                 const float* __restrict__ b, float eps, int d, __nv_bfloat16* __restrict__ y) {
+template <bool LAYERNORM>
+__global__ void __launch_bounds__(kNormThreads)
+add_norm_kernel(__nv_bfloat16* __restrict__ x, const __nv_bfloat16* delta, const float* __restrict__ w,
+                const float* __restrict__ b, float eps, int d, __nv_bfloat16* y) {
   __shared__ float red[32];
-  const __nv_bfloat16* row = x + (size_t)blockIdx.x * d;
+  const int nvec = d >> 3;
+  uint4* xrow = reinterpret_cast<uint4*>(x + (size_t)blockIdx.x * d);
+  const uint4* drow = delta ? reinterpret_cast<const uint4*>(delta + (size_t)blockIdx.x * d) : nullptr;
+  float v[kNormVecs][8];
   float s = 0.0f;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) s += __bfloat162float(row[i]);
-  const float mu = block_sum(s, red) / (float)d;
-  float ss = 0.0f;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    const float c = __bfloat162float(row[i]) - mu;
-    ss += c * c;
+#pragma unroll
+  for (int j = 0; j < kNormVecs; ++j) {
+    const int i = threadIdx.x + j * kNormThreads;
+    if (i < nvec) {
+      uint4 raw = xrow[i];
+      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
+      if (drow) {
+        const uint4 dr = drow[i];
+        const __nv_bfloat162* dh = reinterpret_cast<const __nv_bfloat162*>(&dr);
+        __nv_bfloat162 o[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float2 a = __bfloat1622float2(h[e]), c = __bfloat1622float2(dh[e]);
+          o[e] = __floats2bfloat162_rn(a.x + c.x, a.y + c.y);
+          const float2 r = __bfloat1622float2(o[e]);
+          v[j][2 * e] = r.x; v[j][2 * e + 1] = r.y;
+        }
+        xrow[i] = *reinterpret_cast<const uint4*>(o);
+      } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float2 a = __bfloat1622float2(h[e]);
+          v[j][2 * e] = a.x; v[j][2 * e + 1] = a.y;
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < 8; ++e) s += LAYERNORM ? v[j][e] : v[j][e] * v[j][e];
+    }
   }
-  const float r = rsqrtf(block_sum(ss, red) / (float)d + eps);
-  __nv_bfloat16* out = y + (size_t)blockIdx.x * d;
-  for (int i = threadIdx.x; i < d; i += blockDim.x)
-    out[i] = __float2bfloat16_rn((__bfloat162float(row[i]) - mu) * r * w[i] + b[i]);
+  float mu = 0.0f, r;
+  if (LAYERNORM) {
+    mu = block_sum(s, red) / (float)d;
+    float ss = 0.0f;
+#pragma unroll
+    for (int j = 0; j < kNormVecs; ++j) {
+      if (threadIdx.x + j * kNormThreads < nvec) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { const float c = v[j][e] - mu; ss += c * c; }
+      }
+    }
+    r = rsqrtf(block_sum(ss, red) / (float)d + eps);
+  } else {
+    r = rsqrtf(block_sum(s, red) / (float)d + eps);
+  }
+  uint4* yrow = reinterpret_cast<uint4*>(y + (size_t)blockIdx.x * d);
+#pragma unroll
+  for (int j = 0; j < kNormVecs; ++j) {
+    const int i = threadIdx.x + j * kNormThreads;
+    if (i < nvec) {
+      const float4 w0 = reinterpret_cast<const float4*>(w)[2 * i], w1 = reinterpret_cast<const float4*>(w)[2 * i + 1];
+      const float ww[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+      float bb[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+      if (LAYERNORM) {
+        const float4 b0 = reinterpret_cast<const float4*>(b)[2 * i], b1 = reinterpret_cast<const float4*>(b)[2 * i + 1];
+        bb[0] = b0.x; bb[1] = b0.y; bb[2] = b0.z; bb[3] = b0.w; bb[4] = b1.x; bb[5] = b1.y; bb[6] = b1.z; bb[7] = b1.w;
+      }
+      __nv_bfloat162 o[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        o[e] = __floats2bfloat162_rn((v[j][2 * e] - mu) * r * ww[2 * e] + bb[2 * e],
+                                     (v[j][2 * e + 1] - mu) * r * ww[2 * e + 1] + bb[2 * e + 1]);
+      yrow[i] = *reinterpret_cast<const uint4*>(o);
+    }
+  }
 }
 
 // cos/sin table [max_seq][dh/2] in fp32, evaluated in fp64.
@@ -358,13 +408,16 @@ int launch_embedding(const int32_t* tokens, const __nv_bfloat16* embed, const __
   QZO_LAUNCH(embedding_kernel, dim3(T), dim3(128), 0, st, tokens, embed, pos, S, d, vocab, x);
   return QZO_OK;
 }
-int launch_rmsnorm(const __nv_bfloat16* x, const float* w, float eps, int T, int d, __nv_bfloat16* y, cudaStream_t st) {
-  QZO_LAUNCH(rmsnorm_kernel, dim3(T), dim3(256), 0, st, x, w, eps, d, y);
+int launch_add_rmsnorm(__nv_bfloat16* x, const __nv_bfloat16* delta, const float* w, float eps, int T, int d,
+                       __nv_bfloat16* y, cudaStream_t st) {
+  if ((d % 8) || d > kNormVecs * kNormThreads * 8) return QZO_ERR_BAD_ARG;
+  QZO_LAUNCH(add_norm_kernel<false>, dim3(T), dim3(kNormThreads), 0, st, x, delta, w, nullptr, eps, d, y);
   return QZO_OK;
 }
-int launch_layernorm(const __nv_bfloat16* x, const float* w, const float* b, float eps, int T, int d,
-                     __nv_bfloat16* y, cudaStream_t st) {
-  QZO_LAUNCH(layernorm_kernel, dim3(T), dim3(256), 0, st, x, w, b, eps, d, y);
+int launch_add_layernorm(__nv_bfloat16* x, const __nv_bfloat16* delta, const float* w, const float* b, float eps,
+                         int T, int d, __nv_bfloat16* y, cudaStream_t st) {
+  if ((d % 8) || d > kNormVecs * kNormThreads * 8) return QZO_ERR_BAD_ARG;
+  QZO_LAUNCH(add_norm_kernel<true>, dim3(T), dim3(kNormThreads), 0, st, x, delta, w, b, eps, d, y);
   return QZO_OK;
 }
 int launch_rope_table(float* cs, int max_seq, int dh, float theta, cudaStream_t st) {

@@ -5,9 +5,11 @@
 namespace qzo {
 int launch_embedding(const int32_t* tokens, const __nv_bfloat16* embed, const __nv_bfloat16* pos, int T, int S, int d,
                      int vocab, __nv_bfloat16* x, cudaStream_t st);
-int launch_rmsnorm(const __nv_bfloat16* x, const float* w, float eps, int T, int d, __nv_bfloat16* y, cudaStream_t st);
-int launch_layernorm(const __nv_bfloat16* x, const float* w, const float* b, float eps, int T, int d,
-                     __nv_bfloat16* y, cudaStream_t st);
+// x <- x + delta (skipped when delta is null), then y = norm(x); y may alias delta.
+int launch_add_rmsnorm(__nv_bfloat16* x, const __nv_bfloat16* delta, const float* w, float eps, int T, int d,
+                       __nv_bfloat16* y, cudaStream_t st);
+int launch_add_layernorm(__nv_bfloat16* x, const __nv_bfloat16* delta, const float* w, const float* b, float eps,
+                         int T, int d, __nv_bfloat16* y, cudaStream_t st);
 int launch_rope_table(float* cs, int max_seq, int dh, float theta, cudaStream_t st);
 int launch_rope(__nv_bfloat16* q, __nv_bfloat16* k, int ldq, int ldk, const float* cs, int T, int S, int H, int dh,
                 cudaStream_t st);
@@ -22,10 +24,19 @@ int launch_ddc(const float* lp, const float* lm, float eps, float lr, float clip
 // gemm_w4a16.cu
 int gemm_splits(int M, int K, int N);
 size_t gemm_workspace_bytes(int M, int K, int N);
-int launch_perturbed_gemm(const __nv_bfloat16* d_x, const void* d_wq, const __nv_bfloat16* d_scales,
-                          const float* d_bias, const __nv_bfloat16* d_residual, __nv_bfloat16* d_y, int ldo,
-                          int M, int K, int N, uint64_t seed, uint64_t idx_base, int sign, float eps,
-                          void* d_ws, size_t ws_bytes, int* d_status, cudaStream_t st);
+// One linear of a grouped launch: Y = X W' (+ bias), Y bf16 [M][ldo].
+constexpr int kMaxGroupedLinears = 3;
+struct GemmLinear {
+  const void* wq;                 // kernel-layout int4 weights [K][N]
+  const __nv_bfloat16* scales;    // [G][N]
+  const float* bias;              // [N] or null
+  __nv_bfloat16* out;             // [M][ldo]; 16-byte aligned, ldo a multiple of 8
+  int ldo, N;
+  uint64_t idx_base;              // logical index of scale [0][0]
+};
+int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const GemmLinear* lins, int n_lin,
+                                uint64_t seed, int sign, float eps, void* d_ws, size_t ws_bytes, int* d_status,
+                                cudaStream_t st);
 int launch_bf16_gemm_f32out(const __nv_bfloat16* d_x, const __nv_bfloat16* d_w, float* d_out, int M, int K, int N,
                             int* d_status, cudaStream_t st);
 }  // namespace qzo

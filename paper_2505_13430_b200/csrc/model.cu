@@ -164,23 +164,41 @@ int plan_workspace(const qzo_model_desc& d, int T, WsPlan* p) {
   return QZO_OK;
 }
 
-static int norm(qzo_model* m, const __nv_bfloat16* in, const float* w, const float* b, int T, __nv_bfloat16* out) {
-  if (m->desc.arch == QZO_ARCH_LLAMA) return launch_rmsnorm(in, w, m->desc.norm_eps, T, m->desc.d_model, out, m->stream);
-  return launch_layernorm(in, w, b, m->desc.norm_eps, T, m->desc.d_model, out, m->stream);
+// x += delta (when delta is given), then out = norm(x): the residual add of a block's projection is
+// fused into the norm that follows it.
+static int add_norm(qzo_model* m, __nv_bfloat16* x, const __nv_bfloat16* delta, const float* w, const float* b, int T,
+                    __nv_bfloat16* out) {
+  if (m->desc.arch == QZO_ARCH_LLAMA)
+    return launch_add_rmsnorm(x, delta, w, m->desc.norm_eps, T, m->desc.d_model, out, m->stream);
+  return launch_add_layernorm(x, delta, w, b, m->desc.norm_eps, T, m->desc.d_model, out, m->stream);
 }
 
-static int linear(qzo_model* m, const Linear& L, const __nv_bfloat16* in, const __nv_bfloat16* residual,
-                  __nv_bfloat16* out, int ldo, int T, uint64_t seed, int sign, float eps) {
+// Up to three block linears that read the same input, in one launch.
+static int linears(qzo_model* m, const Linear* const* Ls, __nv_bfloat16* const* outs, int n, int ldo,
+                   const __nv_bfloat16* in, int T, uint64_t seed, int sign, float eps) {
+  GemmLinear g[kMaxGroupedLinears];
+  double flops = 0.0;
+  for (int j = 0; j < n; ++j) {
+    g[j] = GemmLinear{Ls[j]->wq, m->scales + Ls[j]->idx_base, Ls[j]->bias, outs[j], ldo, Ls[j]->N,
+                      (uint64_t)Ls[j]->idx_base};
+    flops += 2.0 * T * (double)Ls[j]->K * (double)Ls[j]->N;
+  }
   const bool timed = m->profiling && m->events_used + 2 <= m->events.size();
   if (timed) QZO_CUDA_TRY(cudaEventRecord(m->events[m->events_used], m->stream));
-  QZO_TRY(launch_perturbed_gemm(in, L.wq, m->scales + L.idx_base, L.bias, residual, out, ldo, T, L.K, L.N, seed,
-                                (uint64_t)L.idx_base, sign, eps, m->gemm_ws, m->gemm_ws_bytes, m->status, m->stream));
+  QZO_TRY(launch_perturbed_gemm_group(in, T, Ls[0]->K, g, n, seed, sign, eps, m->gemm_ws, m->gemm_ws_bytes, m->status,
+                                      m->stream));
   if (timed) {
     QZO_CUDA_TRY(cudaEventRecord(m->events[m->events_used + 1], m->stream));
     m->events_used += 2;
-    m->profiled_flops += 2.0 * T * (double)L.K * (double)L.N;
+    m->profiled_flops += flops;
   }
   return QZO_OK;
+}
+static int linear(qzo_model* m, const Linear& L, const __nv_bfloat16* in, __nv_bfloat16* out, int ldo, int T,
+                  uint64_t seed, int sign, float eps) {
+  const Linear* Ls[1] = {&L};
+  __nv_bfloat16* outs[1] = {out};
+  return linears(m, Ls, outs, 1, ldo, in, T, seed, sign, eps);
 }
 
 int forward_loss(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S, uint64_t seed, int sign,
@@ -190,29 +208,39 @@ int forward_loss(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels,
   cudaStream_t st = m->stream;
   const bool llama = d.arch == QZO_ARCH_LLAMA;
   QZO_TRY(launch_embedding(d_tokens, m->embed, llama ? nullptr : m->pos_embed, T, S, dm, d.vocab, m->x, st));
+  // The residual stream x is updated lazily: a projection writes its output to xn, and the norm that
+  // follows adds it to x before normalising (x += xn; xn = norm(x)).
+  const __nv_bfloat16* pending = nullptr;          // projection output not yet added to x
   for (int li = 0; li < d.n_layers; ++li) {
     const Layer& L = m->layers[li];
-    QZO_TRY(norm(m, m->x, L.norm1_w, L.norm1_b, T, m->xn));
-    for (int j = 0; j < 3; ++j)
-      QZO_TRY(linear(m, L.lin[j], m->xn, nullptr, m->qkv + (size_t)j * dm, 3 * dm, T, seed, sign, eps));
+    QZO_TRY(add_norm(m, m->x, pending, L.norm1_w, L.norm1_b, T, m->xn));
+    if (li > 0 && li - 1 == m->capture_layer)
+      QZO_CUDA_TRY(cudaMemcpyAsync(m->capture, m->x, (size_t)T * dm * 2, cudaMemcpyDeviceToDevice, st));
+    {
+      const Linear* qkv_l[3] = {&L.lin[0], &L.lin[1], &L.lin[2]};
+      __nv_bfloat16* qkv_o[3] = {m->qkv, m->qkv + dm, m->qkv + 2 * dm};
+      QZO_TRY(linears(m, qkv_l, qkv_o, 3, 3 * dm, m->xn, T, seed, sign, eps));
+    }
     if (llama) QZO_TRY(launch_rope(m->qkv, m->qkv + dm, 3 * dm, 3 * dm, m->rope_cs, T, S, H, dh, st));
     QZO_TRY(launch_attention(m->qkv, m->qkv + dm, m->qkv + 2 * dm, 3 * dm, 3 * dm, 3 * dm, m->att, dm, B, S, H, dh, st));
-    QZO_TRY(linear(m, L.lin[3], m->att, m->x, m->x, dm, T, seed, sign, eps));
-    QZO_TRY(norm(m, m->x, L.norm2_w, L.norm2_b, T, m->xn));
+    QZO_TRY(linear(m, L.lin[3], m->att, m->xn, dm, T, seed, sign, eps));
+    QZO_TRY(add_norm(m, m->x, m->xn, L.norm2_w, L.norm2_b, T, m->xn));
     if (llama) {
-      QZO_TRY(linear(m, L.lin[4], m->xn, nullptr, m->mlp_a, F, T, seed, sign, eps));
-      QZO_TRY(linear(m, L.lin[5], m->xn, nullptr, m->mlp_b, F, T, seed, sign, eps));
+      const Linear* gu_l[2] = {&L.lin[4], &L.lin[5]};
+      __nv_bfloat16* gu_o[2] = {m->mlp_a, m->mlp_b};
+      QZO_TRY(linears(m, gu_l, gu_o, 2, F, m->xn, T, seed, sign, eps));
       QZO_TRY(launch_silu_mul(m->mlp_a, m->mlp_b, m->mlp_a, (int64_t)T * F, st));
-      QZO_TRY(linear(m, L.lin[6], m->mlp_a, m->x, m->x, dm, T, seed, sign, eps));
+      QZO_TRY(linear(m, L.lin[6], m->mlp_a, m->xn, dm, T, seed, sign, eps));
     } else {
-      QZO_TRY(linear(m, L.lin[4], m->xn, nullptr, m->mlp_a, F, T, seed, sign, eps));
+      QZO_TRY(linear(m, L.lin[4], m->xn, m->mlp_a, F, T, seed, sign, eps));
       QZO_TRY(launch_relu(m->mlp_a, (int64_t)T * F, st));
-      QZO_TRY(linear(m, L.lin[5], m->mlp_a, m->x, m->x, dm, T, seed, sign, eps));
+      QZO_TRY(linear(m, L.lin[5], m->mlp_a, m->xn, dm, T, seed, sign, eps));
     }
-    if (li == m->capture_layer)
-      QZO_CUDA_TRY(cudaMemcpyAsync(m->capture, m->x, (size_t)T * dm * 2, cudaMemcpyDeviceToDevice, st));
+    pending = m->xn;
   }
-  QZO_TRY(norm(m, m->x, m->final_norm_w, m->final_norm_b, T, m->xn));
+  QZO_TRY(add_norm(m, m->x, pending, m->final_norm_w, m->final_norm_b, T, m->xn));
+  if (d.n_layers - 1 == m->capture_layer)
+    QZO_CUDA_TRY(cudaMemcpyAsync(m->capture, m->x, (size_t)T * dm * 2, cudaMemcpyDeviceToDevice, st));
   QZO_TRY(launch_bf16_gemm_f32out(m->xn, m->lm_head, m->logits, T, dm, d.vocab, m->status, st));
   QZO_TRY(launch_cross_entropy(m->logits, d_labels, T, d.vocab, m->row_loss, d_loss, st));
   m->last_T = T;
@@ -325,12 +353,16 @@ int qzo_perturbed_gemm(const void* d_x_bf16, const void* d_wq, const void* d_sca
                        float eps, void* d_workspace, size_t workspace_bytes, int* d_status, void* stream) {
   if (!d_x_bf16 || !d_wq || !d_scales_bf16 || !d_y_bf16) return QZO_ERR_BAD_ARG;
   if (sign < -1 || sign > 1 || !(eps > 0.0f)) return QZO_ERR_BAD_ARG;
-  if (((uintptr_t)d_x_bf16 & 15) || ((uintptr_t)d_wq & 15) || ((uintptr_t)d_scales_bf16 & 15)) return QZO_ERR_BAD_ARG;
+  if (((uintptr_t)d_x_bf16 & 15) || ((uintptr_t)d_wq & 15) || ((uintptr_t)d_scales_bf16 & 15) ||
+      ((uintptr_t)d_y_bf16 & 15))
+    return QZO_ERR_BAD_ARG;
   if (d_workspace && ((uintptr_t)d_workspace & 255)) return QZO_ERR_WORKSPACE;
   QZO_TRY(check_device());
-  return launch_perturbed_gemm((const __nv_bfloat16*)d_x_bf16, d_wq, (const __nv_bfloat16*)d_scales_bf16, d_bias,
-                               nullptr, (__nv_bfloat16*)d_y_bf16, N, M, K, N, seed, scale_index_base, sign, eps,
-                               d_workspace, workspace_bytes, d_status, (cudaStream_t)stream);
+  if (N <= 0 || (N % 8)) return QZO_ERR_BAD_ARG;
+  const GemmLinear g{d_wq, (const __nv_bfloat16*)d_scales_bf16, d_bias, (__nv_bfloat16*)d_y_bf16, N, N,
+                     scale_index_base};
+  return launch_perturbed_gemm_group((const __nv_bfloat16*)d_x_bf16, M, K, &g, 1, seed, sign, eps, d_workspace,
+                                     workspace_bytes, d_status, (cudaStream_t)stream);
 }
 
 int qzo_update_scales_flat(void* d_scales_bf16, int64_t count, uint64_t seed, uint64_t index_base, float lr, float g,

@@ -2,9 +2,9 @@
 
     python -m paper_2505_13430_b200.gemm_sweep [--shapes KxN,...] [--tokens M,...] [--iters I] [--json]
 
-For every shape it times qzo_perturbed_gemm with CUDA events, rotating through enough distinct
-weight / scale / activation sets that every launch streams its operands from HBM (the rotation
-exceeds the L2 capacity), and prints the achieved fraction of the roofline
+For every shape it times qzo_perturbed_gemm with CUDA events around replays of a CUDA graph that
+holds `iters` launches, rotating through enough distinct weight / scale / activation sets that
+every launch streams its operands from HBM (the rotation exceeds the L2 capacity), and prints the achieved fraction of the roofline
 max(bytes / HBM bandwidth, flops / dense bf16 peak) with
 bytes = K N / 2 + 2 ceil(K/128) N + 2 M K + 2 M N and flops = 2 M K N.
 """
@@ -32,7 +32,7 @@ def gemm_bytes(M, K, N):
     return K * N // 2 + 2 * ((K + 127) // 128) * N + 2 * M * K + 2 * M * N
 
 
-def run_shape(M, K, N, iters, sign=1):
+def run_shape(M, K, N, iters, sign=1, reps=5):
     per_set = gemm_bytes(M, K, N)
     n_sets = max(2, min(64, (2 * L2_BYTES) // per_set + 1))
     sets = []
@@ -44,6 +44,7 @@ def run_shape(M, K, N, iters, sign=1):
         y = torch.empty((M, N), device="cuda", dtype=torch.bfloat16)
         sets.append((x, wq, s, y))
         del words
+    iters = max(iters, n_sets)
     need = qzo.qzo_gemm_workspace_bytes(M, K, N)
     ws = torch.empty((max(need, 256),), dtype=torch.uint8, device="cuda")
     status = torch.zeros((1,), dtype=torch.int32, device="cuda")
@@ -55,14 +56,24 @@ def run_shape(M, K, N, iters, sign=1):
     for i in range(max(3, n_sets)):
         call(i)
     torch.cuda.synchronize()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record()
-    for i in range(iters):
-        call(i)
-    ev1.record()
-    torch.cuda.synchronize()
+    # The launches of one timed pass are recorded into a CUDA graph and replayed, so that the
+    # figure is device time: at small M a launch from Python costs more than the kernel runs.
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            for i in range(iters):
+                call(i)
+        graph.replay()
+        side.synchronize()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(side)
+        for _ in range(reps):
+            graph.replay()
+        ev1.record(side)
+        side.synchronize()
     assert int(status.item()) == 0
-    return ev0.elapsed_time(ev1) * 1e3 / iters, n_sets      # microseconds
+    return ev0.elapsed_time(ev1) * 1e3 / (iters * reps), n_sets      # microseconds per launch
 
 
 def main():
