@@ -108,6 +108,27 @@ int qzo_perturbed_gemm(const void* d_x_bf16, const void* d_wq, const void* d_sca
                        uint64_t seed, uint64_t scale_index_base, int sign, float eps,
                        void* d_workspace, size_t workspace_bytes, int* d_status, void* stream);
 
+/* The same linear for callers that must not allocate device memory and have no workspace to
+ * lend: for example a serving process that gave all device memory to its own pool when it
+ * started, or a latency-critical loop in which the device-wide synchronisation of an allocation
+ * is not acceptable.  (The paper has no counterpart; this is a property of the library.)
+ * Arguments and result are those of qzo_perturbed_gemm without the workspace.  The split-K
+ * partial sums go to a fixed array of QZO_NOALLOC_SCRATCH_BYTES inside the library image: every
+ * device that loads the library holds that much until the process exits.  The call allocates
+ * nothing: no cudaMalloc, no cudaFree, no allocating library routine.
+ *  - A problem whose partial sums (qzo_gemm_workspace_bytes) exceed the array returns
+ *    QZO_ERR_WORKSPACE and launches nothing.
+ *  - The first call on each device looks the array's device address up (with that device
+ *    current); make that first call before any stream capture begins.
+ *  - All calls on a device share the one array, which keeps the last call's partial sums (none
+ *    of it needs clearing: each call overwrites every element it later reads).  Two calls that
+ *    overlap on the GPU (different streams) race on it; keep them on one stream or order them. */
+#define QZO_NOALLOC_SCRATCH_BYTES (16u << 20)
+int qzo_perturbed_gemm_noalloc(const void* d_x_bf16, const void* d_wq, const void* d_scales_bf16,
+                               const float* d_bias, void* d_y_bf16, int M, int K, int N,
+                               uint64_t seed, uint64_t scale_index_base, int sign, float eps,
+                               int* d_status, void* stream);
+
 /* Seeded update of a flat run of scales (Algorithm 1, last loop, with Eq. 6 applied to g):
  *   s_i <- bf16(max(s_i - (lr clip(g,-C,C)) z_i, 0)), i = index_base .. index_base+count-1.
  * d_scales bf16 [count], in place.  g must be finite, clip >= 0. */

@@ -860,3 +860,58 @@ int launch_bf16_gemm_f32out(const __nv_bfloat16* d_x, const __nv_bfloat16* d_w, 
 }
 
 }  // namespace qzo
+
+// ------------------------------------------------------------------------------------------
+// Entry point that allocates nothing: the split-K partial sums live in a fixed array inside
+// the library image instead of a caller-provided workspace.
+// ------------------------------------------------------------------------------------------
+namespace {
+
+// Scratch of the allocation-free entry point.  One copy per device that loads the library,
+// held until the process exits.  In host code this name is only a handle for the symbol, not a
+// device address: the address is resolved per device below and passed to the kernels.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[QZO_NOALLOC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_noalloc_mutex;
+void* g_noalloc_ptr[kMaxDevices] = {};
+
+// Device address of the scratch array on the current device (resolved once per device).
+int noalloc_scratch_address(void** out) {
+  int dev = 0;
+  QZO_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return QZO_ERR_UNSUPPORTED_DEVICE;
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  if (g_noalloc_ptr[dev] == nullptr) {
+    void* ptr = nullptr;
+    QZO_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_noalloc_scratch));
+    if (ptr == nullptr) return QZO_ERR_CUDA;
+    g_noalloc_ptr[dev] = ptr;
+  }
+  *out = g_noalloc_ptr[dev];
+  return QZO_OK;
+}
+
+}  // namespace
+
+extern "C" int qzo_perturbed_gemm_noalloc(const void* d_x_bf16, const void* d_wq, const void* d_scales_bf16,
+                                          const float* d_bias, void* d_y_bf16, int M, int K, int N, uint64_t seed,
+                                          uint64_t scale_index_base, int sign, float eps, int* d_status,
+                                          void* stream) {
+  if (!d_x_bf16 || !d_wq || !d_scales_bf16 || !d_y_bf16) return QZO_ERR_BAD_ARG;
+  if (M <= 0 || K <= 0 || N <= 0 || (N % 8) || (K % 8)) return QZO_ERR_BAD_ARG;
+  if (sign < -1 || sign > 1 || !(eps > 0.0f)) return QZO_ERR_BAD_ARG;
+  if (((uintptr_t)d_x_bf16 & 15) || ((uintptr_t)d_wq & 15) || ((uintptr_t)d_scales_bf16 & 15) ||
+      ((uintptr_t)d_y_bf16 & 15))
+    return QZO_ERR_BAD_ARG;
+  // a problem whose partial sums do not fit the fixed array is refused, never truncated
+  if (qzo::gemm_workspace_bytes(M, K, N) > (size_t)QZO_NOALLOC_SCRATCH_BYTES) return QZO_ERR_WORKSPACE;
+  QZO_TRY(qzo::check_device());
+  void* scratch = nullptr;
+  QZO_TRY(noalloc_scratch_address(&scratch));
+  const qzo::GemmLinear g{d_wq, (const __nv_bfloat16*)d_scales_bf16, d_bias, (__nv_bfloat16*)d_y_bf16, N, N,
+                          scale_index_base};
+  return qzo::launch_perturbed_gemm_group((const __nv_bfloat16*)d_x_bf16, M, K, &g, 1, seed, sign, eps, scratch,
+                                          (size_t)QZO_NOALLOC_SCRATCH_BYTES, d_status, (cudaStream_t)stream);
+}
+

@@ -23,7 +23,7 @@ DTYPE_U32 = 2
 EXPORTS = (
     "qzo_strerror", "qzo_last_cuda_error", "qzo_philox_words", "qzo_normals", "qzo_quantize_int4",
     "qzo_unpack_int4", "qzo_repacked_bytes", "qzo_repack_int4", "qzo_unpack_kernel_layout",
-    "qzo_gemm_workspace_bytes", "qzo_perturbed_gemm", "qzo_update_scales_flat", "qzo_num_scales",
+    "qzo_gemm_workspace_bytes", "qzo_perturbed_gemm", "qzo_perturbed_gemm_noalloc", "qzo_update_scales_flat", "qzo_num_scales",
     "qzo_scale_layout", "qzo_workspace_bytes", "qzo_init_model", "qzo_free_model", "qzo_forward_loss",
     "qzo_update_scales", "qzo_step", "qzo_step_host", "qzo_debug_set_capture", "qzo_debug_layer_output",
     "qzo_device_status", "qzo_launch_count", "qzo_profile_gemms", "qzo_profile_read",
@@ -72,6 +72,7 @@ def _load():
         "qzo_unpack_kernel_layout": (ci, [vp, ci, ci, vp, vp]),
         "qzo_gemm_workspace_bytes": (ci, [ci, ci, ci, P(sz)]),
         "qzo_perturbed_gemm": (ci, [vp, vp, vp, vp, vp, ci, ci, ci, u64, u64, ci, cf, vp, sz, vp, vp]),
+        "qzo_perturbed_gemm_noalloc": (ci, [vp, vp, vp, vp, vp, ci, ci, ci, u64, u64, ci, cf, vp, vp]),
         "qzo_update_scales_flat": (ci, [vp, i64, u64, u64, cf, cf, cf, vp]),
         "qzo_num_scales": (ci, [P(ModelDesc), P(i64), P(i64)]),
         "qzo_scale_layout": (ci, [P(ModelDesc), ci, ci, P(i64), P(ci), P(ci)]),
@@ -193,6 +194,19 @@ def qzo_perturbed_gemm(x, wq, scales, M, K, N, seed, scale_index_base, sign, eps
     _check(_lib.qzo_perturbed_gemm(_ptr(x), _ptr(wq), _ptr(scales), _ptr(bias), _ptr(y), M, K, N, seed,
                                    scale_index_base, sign, eps, _ptr(workspace), ws_bytes, _ptr(status), _stream()),
            "qzo_perturbed_gemm")
+    return y
+
+
+NOALLOC_SCRATCH_BYTES = 16 << 20
+
+
+def qzo_perturbed_gemm_noalloc(x, wq, scales, y, M, K, N, seed, scale_index_base, sign, eps, bias=None, status=None):
+    """qzo_perturbed_gemm for callers that cannot allocate: no workspace argument (the library's
+    fixed scratch array is used) and the output tensor y is the caller's.  Nothing is allocated here."""
+    _cuda(x, torch.bfloat16), _cuda(wq, torch.uint8), _cuda(scales, torch.bfloat16), _cuda(y, torch.bfloat16)
+    _check(_lib.qzo_perturbed_gemm_noalloc(_ptr(x), _ptr(wq), _ptr(scales), _ptr(bias), _ptr(y), M, K, N, seed,
+                                           scale_index_base, sign, eps, _ptr(status), _stream()),
+           "qzo_perturbed_gemm_noalloc")
     return y
 
 
