@@ -158,29 +158,33 @@ __global__ void rope_table_kernel(float* __restrict__ cs, int max_seq, int half,
   cs[2 * idx + 1] = (float)s;
 }
 
-// Rotate pairs (i, i + dh/2) of q and k, in place.  q at buf[t][q_off + h*dh + .], k at k_off.
+// Rotate pairs (i, i + dh/2) of q and k, in place.  q at buf[t][h*dh + .] with row stride ldq, k
+// likewise.  One thread rotates eight consecutive pairs of one head of q or of k (16-byte accesses).
 __global__ void rope_kernel(__nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ k, int ldq, int ldk,
                             const float* __restrict__ cs, int S, int H, int dh, int64_t total) {
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= total) return;
   const int half = dh / 2;
-  const int i = (int)(idx % half);
-  const int h = (int)((idx / half) % H);
-  const int t = (int)(idx / ((int64_t)half * H));
+  const int vecs = half / 8;                       // 8-pair groups per head
+  const int v = (int)(idx % vecs);
+  const int h = (int)((idx / vecs) % H);
+  const int which = (int)((idx / ((int64_t)vecs * H)) & 1);
+  const int t = (int)(idx / ((int64_t)vecs * H * 2));
   const int pos = t % S;
-  const float c = cs[2 * (pos * half + i)], s = cs[2 * (pos * half + i) + 1];
-  {
-    __nv_bfloat16* p = q + (size_t)t * ldq + h * dh + i;
-    const float a = __bfloat162float(p[0]), b = __bfloat162float(p[half]);
-    p[0] = __float2bfloat16_rn(a * c - b * s);
-    p[half] = __float2bfloat16_rn(b * c + a * s);
+  __nv_bfloat16* p = (which ? k + (size_t)t * ldk : q + (size_t)t * ldq) + h * dh + v * 8;
+  uint4 lo = *reinterpret_cast<const uint4*>(p), hi = *reinterpret_cast<const uint4*>(p + half);
+  __nv_bfloat162* a2 = reinterpret_cast<__nv_bfloat162*>(&lo);
+  __nv_bfloat162* b2 = reinterpret_cast<__nv_bfloat162*>(&hi);
+  const float4* c4 = reinterpret_cast<const float4*>(cs + 2 * ((size_t)pos * half + v * 8));   // {cos, sin} pairs
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float4 cs01 = c4[e];                     // cos0 sin0 cos1 sin1
+    const float2 a = __bfloat1622float2(a2[e]), b = __bfloat1622float2(b2[e]);
+    a2[e] = __floats2bfloat162_rn(a.x * cs01.x - b.x * cs01.y, a.y * cs01.z - b.y * cs01.w);
+    b2[e] = __floats2bfloat162_rn(b.x * cs01.x + a.x * cs01.y, b.y * cs01.z + a.y * cs01.w);
   }
-  {
-    __nv_bfloat16* p = k + (size_t)t * ldk + h * dh + i;
-    const float a = __bfloat162float(p[0]), b = __bfloat162float(p[half]);
-    p[0] = __float2bfloat16_rn(a * c - b * s);
-    p[half] = __float2bfloat16_rn(b * c + a * s);
-  }
+  *reinterpret_cast<uint4*>(p) = lo;
+  *reinterpret_cast<uint4*>(p + half) = hi;
 }
 
 // Causal attention with online softmax on the legacy tensor-core path (mma.sync m16n8k16,
@@ -339,19 +343,32 @@ attention_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
   }
 }
 
-// act = silu(gate) * up
+// act = silu(gate) * up, eight elements per thread (n is a multiple of 8)
 __global__ void silu_mul_kernel(const __nv_bfloat16* __restrict__ gate, const __nv_bfloat16* __restrict__ up,
-                                __nv_bfloat16* __restrict__ out, int64_t n) {
+                                __nv_bfloat16* __restrict__ out, int64_t nvec) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n) return;
-  const float g = __bfloat162float(gate[i]), u = __bfloat162float(up[i]);
-  out[i] = __float2bfloat16_rn(g / (1.0f + __expf(-g)) * u);
+  if (i >= nvec) return;
+  const uint4 g4 = reinterpret_cast<const uint4*>(gate)[i], u4 = reinterpret_cast<const uint4*>(up)[i];
+  const __nv_bfloat162* g2 = reinterpret_cast<const __nv_bfloat162*>(&g4);
+  const __nv_bfloat162* u2 = reinterpret_cast<const __nv_bfloat162*>(&u4);
+  __nv_bfloat162 o[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float2 g = __bfloat1622float2(g2[e]), u = __bfloat1622float2(u2[e]);
+    o[e] = __floats2bfloat162_rn(g.x / (1.0f + __expf(-g.x)) * u.x, g.y / (1.0f + __expf(-g.y)) * u.y);
+  }
+  reinterpret_cast<uint4*>(out)[i] = *reinterpret_cast<const uint4*>(o);
 }
 
-__global__ void relu_kernel(__nv_bfloat16* __restrict__ x, int64_t n) {
+__global__ void relu_kernel(__nv_bfloat16* __restrict__ x, int64_t nvec) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n) return;
-  x[i] = __float2bfloat16_rn(fmaxf(__bfloat162float(x[i]), 0.0f));
+  if (i >= nvec) return;
+  uint4 v = reinterpret_cast<uint4*>(x)[i];
+  __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&v);
+  const __nv_bfloat162 zero = __floats2bfloat162_rn(0.0f, 0.0f);
+#pragma unroll
+  for (int e = 0; e < 4; ++e) h[e] = __hmax2(h[e], zero);
+  reinterpret_cast<uint4*>(x)[i] = v;
 }
 
 // Row-wise cross entropy on fp32 logits: row_loss[t] = logsumexp(logits[t]) - logits[t][label],
@@ -427,7 +444,8 @@ int launch_rope_table(float* cs, int max_seq, int dh, float theta, cudaStream_t 
 }
 int launch_rope(__nv_bfloat16* q, __nv_bfloat16* k, int ldq, int ldk, const float* cs, int T, int S, int H, int dh,
                 cudaStream_t st) {
-  const int64_t total = (int64_t)T * H * (dh / 2);
+  if ((dh % 16) || (ldq % 8) || (ldk % 8)) return QZO_ERR_BAD_ARG;
+  const int64_t total = (int64_t)T * 2 * H * (dh / 16);
   QZO_LAUNCH(rope_kernel, dim3((unsigned)ceil_div64(total, 256)), dim3(256), 0, st, q, k, ldq, ldk, cs, S, H, dh, total);
   return QZO_OK;
 }
@@ -452,11 +470,13 @@ int launch_attention(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_
   return QZO_OK;
 }
 int launch_silu_mul(const __nv_bfloat16* gate, const __nv_bfloat16* up, __nv_bfloat16* out, int64_t n, cudaStream_t st) {
-  QZO_LAUNCH(silu_mul_kernel, dim3((unsigned)ceil_div64(n, 256)), dim3(256), 0, st, gate, up, out, n);
+  if (n % 8) return QZO_ERR_BAD_ARG;
+  QZO_LAUNCH(silu_mul_kernel, dim3((unsigned)ceil_div64(n / 8, 256)), dim3(256), 0, st, gate, up, out, n / 8);
   return QZO_OK;
 }
 int launch_relu(__nv_bfloat16* x, int64_t n, cudaStream_t st) {
-  QZO_LAUNCH(relu_kernel, dim3((unsigned)ceil_div64(n, 256)), dim3(256), 0, st, x, n);
+  if (n % 8) return QZO_ERR_BAD_ARG;
+  QZO_LAUNCH(relu_kernel, dim3((unsigned)ceil_div64(n / 8, 256)), dim3(256), 0, st, x, n / 8);
   return QZO_OK;
 }
 int launch_cross_entropy(const float* logits, const int32_t* labels, int T, int V, float* row_loss, float* loss,
