@@ -29,3 +29,25 @@ def perturbed_linear(x, q, s, seed, index_base, sign, eps, bias=None):
     if bias is not None:
         y = y + np.asarray(bias, dtype=np.float64)[None, :]
     return y
+
+
+def perturbed_linear_samples(x_rows, q_cols, s_cols, cols, N, seed, index_base, sign, eps, bias_cols=None):
+    """The same Y (Eq. 4 inside Eq. 5) for a few columns `cols` of a layer with N output features.
+
+    x_rows [R][K], q_cols [K][C] and s_cols [G][C] hold the sampled rows / columns only; the
+    logical index of scale (g, cols[c]) is still index_base + g*N + cols[c].  Returns [R][C].
+    """
+    x = np.asarray(x_rows, dtype=np.float64)
+    q = np.asarray(q_cols)
+    sp = np.asarray(s_cols, dtype=np.float64).copy()
+    cols = np.asarray(cols, dtype=np.uint64)
+    K, G = q.shape[0], sp.shape[0]
+    if sign != 0:
+        idx = np.uint64(index_base) + np.arange(G, dtype=np.uint64)[:, None] * np.uint64(N) + cols[None, :]
+        z = philox.normal_from_index(seed, idx).astype(np.float64)
+        sp = sp + float(sign) * float(eps) * z
+    w = sp[np.arange(K) // GROUP] * q.astype(np.float64)
+    y = x @ w
+    if bias_cols is not None:
+        y = y + np.asarray(bias_cols, dtype=np.float64)[None, :]
+    return y

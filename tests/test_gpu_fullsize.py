@@ -1,0 +1,99 @@
+"""GPU parity at the full benchmark sizes, on sampled outputs the oracle computes one by one.
+
+* The standalone perturbed W4A16 GEMM on every K x N and token count of the sweep, in the launch
+  configuration the sweep times (same entry point, same tile / split-K choice): sampled rows and
+  columns (first and last tile, ragged edges, random ones) against the oracle, max relative 2e-2.
+* One full-width decoder block of the Llama-2-7B shape at the benchmark's batch (16 x 256 tokens,
+  so the grouped q/k/v and gate/up launches and the 256-token tiles are the ones the benchmark
+  runs): block output and logits of sampled sequences against the oracle (sequences of a batch do
+  not interact, so the oracle needs only those sequences).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import int4, linear as olinear, model as omodel
+from paper_2505_13430_b200 import inputs
+from tests.helpers import build_oracle_model
+
+pytestmark = pytest.mark.gpu
+
+TOL = 2e-2
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2505_13430_b200 import qzo
+    return qzo
+
+
+def _sample(rng, n, fixed, count):
+    picks = sorted(set([v for v in fixed if 0 <= v < n] + [int(v) for v in rng.integers(0, n, size=count)]))
+    return picks
+
+
+@pytest.mark.parametrize("K,N", inputs.GEMM_SWEEP_KN)
+@pytest.mark.parametrize("M", inputs.GEMM_SWEEP_M)
+def test_sweep_shapes_match_oracle_on_sampled_outputs(lib, M, K, N):
+    g = torch.Generator(device="cuda")
+    g.manual_seed(K * 31 + N * 7 + M)
+    x = torch.randn((M, K), generator=g, device="cuda", dtype=torch.float32).bfloat16()
+    words = torch.randint(-2 ** 31, 2 ** 31 - 1, (K // 8, N), generator=g, device="cuda", dtype=torch.int32)
+    G = (K + 127) // 128
+    s = (torch.rand((G, N), generator=g, device="cuda", dtype=torch.float32) * 0.015 + 0.005).bfloat16()
+    wq = lib.qzo_repack_int4(words, K, N)
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    rng = np.random.default_rng(M + K + N)
+    rows = _sample(rng, M, [0, 1, 15, 16, 127, 128, 255, 256, M - 1], 6)
+    cols = _sample(rng, N, [0, 1, 127, 128, N - 129, N - 128, N - 1], 24)
+    seed, base, eps = 4242 + M, 8 * (N % 7), 1e-3
+    xr = x[rows].float().cpu().numpy()
+    qc = int4.unpack_int4(words[:, cols].cpu().numpy().view(np.uint32))
+    sc = s[:, cols].float().cpu().numpy()
+    for sign in (+1, -1):
+        y = lib.qzo_perturbed_gemm(x, wq, s, M, K, N, seed, base, sign, eps, status=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0, "a bounded device-side wait expired"
+        got = y[rows][:, cols].float().cpu().numpy().astype(np.float64)
+        ref = olinear.perturbed_linear_samples(xr, qc, sc, cols, N, seed, base, sign, eps)
+        assert np.abs(got - ref).max() <= TOL * np.abs(ref).max(), (M, K, N, sign)
+        assert bool(torch.isfinite(y.float()).all())
+
+
+def test_full_width_llama7b_block_matches_oracle_on_sampled_sequences(lib):
+    c = inputs.CONFIGS["llama7b"]
+    cfg = inputs.model_cfg("llama7b", n_layers=1)
+    raw = inputs.raw_model_tensors(cfg, seed=1000)
+    om = build_oracle_model(raw)
+    quant = {(0, name): (torch.from_numpy(int4.pack_int4(om["layers"][0]["lin"][name]["q"]).view(np.int32)),
+                         torch.from_numpy(om["layers"][0]["lin"][name]["s"]).bfloat16())
+             for name in omodel.LINEAR_ORDER["llama"]}
+    B, S = c["batch"], c["seq"]
+    gm = lib.build_model_from_raw(raw, B * S, quantized=quant)
+    del raw
+    tok, lab = inputs.tokens_and_labels(cfg, B, S, seed=7)
+    gm.qzo_debug_set_capture(0)
+    seed, eps = 42, c["eps"]
+    for sign, picks in ((+1, (0, B - 1)), (-1, (B - 1,))):
+        gm.qzo_forward_loss(tok.cuda(), lab.cuda(), seed, sign, eps)
+        hid = gm.qzo_debug_layer_output(0, 0, B * S).view(B, S, -1)
+        logits = gm.qzo_debug_layer_output(0, 1, B * S).view(B, S, -1)
+        assert gm.qzo_device_status() == 0
+        for b in picks:
+            cap = {}
+            omodel.forward_loss(om, tok[b:b + 1].numpy(), lab[b:b + 1].numpy(), seed, sign, eps, capture=cap)
+            ref_h = cap["hidden"][0].reshape(S, -1)
+            got_h = hid[b].float().cpu().numpy().astype(np.float64)
+            assert np.abs(got_h - ref_h).max() <= TOL * np.abs(ref_h).max(), (sign, b)
+            ref_l = cap["logits"].reshape(S, -1)
+            got_l = logits[b].float().cpu().numpy().astype(np.float64)
+            assert np.abs(got_l - ref_l).max() <= TOL * np.abs(ref_l).max(), (sign, b)
+    # whole-batch properties that hold at any size: run-to-run bit determinism of the loss, and a
+    # step with C = 0 (d' = 0) leaves every scale bit-identical
+    l1 = gm.qzo_forward_loss(tok.cuda(), lab.cuda(), seed, +1, eps).cpu().clone()
+    l2 = gm.qzo_forward_loss(tok.cuda(), lab.cuda(), seed, +1, eps).cpu().clone()
+    assert torch.equal(l1.view(torch.int32), l2.view(torch.int32)) and torch.isfinite(l1).all()
+    before = gm.scales.clone()
+    out = gm.qzo_step(tok.cuda(), lab.cuda(), seed, eps, c["lr"], 0.0)
+    assert out[3] == 0.0 and torch.equal(gm.scales.view(torch.int16), before.view(torch.int16))
+    gm.close()

@@ -55,3 +55,24 @@ def test_no_clamp_on_perturbed_scales():
     s = np.full((1, 8), 1e-6, dtype=np.float32)
     sp = linear.perturbed_scales(s, 3, 0, +1, 1e-3)
     assert (sp < 0).any()          # Algorithm 1's PERTURB_SCALES has no max(., 0)
+
+
+def test_sampled_columns_equal_the_full_layer():
+    # perturbed_linear_samples must give the very entries of the full result, with the scale index of
+    # column n still index_base + g*N + n (a shifted or compacted index would draw other z)
+    x, q, s = _case(M=6, K=400, N=24, seed=3)
+    seed, base, eps = 5, 16, 2e-3
+    rows, cols = [0, 3, 5], [0, 7, 23, 11]
+    for sign in (+1, -1, 0):
+        full = linear.perturbed_linear(x, q, s, seed, base, sign, eps)
+        part = linear.perturbed_linear_samples(x[rows], q[:, cols], s[:, cols], cols, 24, seed, base, sign, eps)
+        np.testing.assert_allclose(part, full[np.ix_(rows, cols)], rtol=1e-13, atol=1e-13)
+    # and by brute force for one entry
+    t, n = 3, 23
+    acc = 0.0
+    for k in range(400):
+        g = k // 128
+        z = float(philox.normal_from_index(seed, np.array([base + g * 24 + n]))[0])
+        acc += x[t, k] * (float(s[g, n]) + eps * z) * int(q[k, n])
+    got = linear.perturbed_linear_samples(x[[t]], q[:, [n]], s[:, [n]], [n], 24, seed, base, +1, eps)[0, 0]
+    assert abs(acc - got) <= 1e-12 * max(1.0, abs(acc))
