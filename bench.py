@@ -167,7 +167,7 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2505_13430_b200 import inputs, qzo
+    from paper_2505_13430_b200 import inputs, qzo, replicas
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -181,8 +181,9 @@ def main():
     c = inputs.CONFIGS[workload]
     cfg = inputs.model_cfg(workload)
     B, S = c["batch"], c["seq"]
-    model = qzo.build_random_model_gpu(cfg, B * S, seed=1000 + rank)
-    tok, lab = inputs.tokens_and_labels(cfg, B, S, seed=7 + rank)
+    model_seed, token_seed = replicas.rank_seeds(1000, 7, rank)
+    model = qzo.build_random_model_gpu(cfg, B * S, seed=model_seed)
+    tok, lab = inputs.tokens_and_labels(cfg, B, S, seed=token_seed)
     tok_pin, lab_pin = tok.contiguous().pin_memory(), lab.contiguous().pin_memory()
     tok_d, lab_d = tok.cuda(), lab.cuda()
     n_gemm = cfg["n_layers"] * len(inputs.linear_shapes(cfg)) * 2
@@ -202,12 +203,7 @@ def main():
             fn(t)
         ev1.record(stream)
         barrier()
-        ms = ev0.elapsed_time(ev1)
-        if world > 1:
-            tt = torch.tensor([ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            ms = float(tt.item())
-        return ms
+        return replicas.max_over_ranks(ev0.elapsed_time(ev1), device="cuda")
 
     seed0 = 42
     for t in range(args.warmup):
@@ -239,8 +235,8 @@ def main():
         return
 
     peaks = measured_peaks()
-    value = world * args.steps / (ms / 1000.0)
-    e2e = world * args.steps / (e2e_ms / 1000.0)
+    value = replicas.whole_job_rate(args.steps, world, ms)
+    e2e = replicas.whole_job_rate(args.steps, world, e2e_ms)
     achieved = gemm_flops / (gemm_ms / 1000.0) / 1e12 if gemm_ms > 0 else 0.0
     peak = peaks["bf16_tflops_sustained"]
     line = {"metric": "qzo_steps_per_s", "value": value, "unit": "steps/s", "n_gpus": world, "steps": args.steps,
@@ -254,7 +250,7 @@ def main():
                          "peak_source": f"{peaks['source']} bf16 sustained", "traffic": None,
                          "launches": int(n_l), "gemm_share_of_step": gemm_ms / ms if ms > 0 else None}}
     if not args.no_cpu_baseline:
-        v, cores, desc = oracle_sample(workload)
+        v, cores, desc = oracle_sample(workload, n_seq=8)
         line["cpu_baseline"] = {"value": v, "unit": "steps/s", "cores": cores, "kind": "oracle", "sample": desc}
     print(json.dumps(line))
     if world > 1:
