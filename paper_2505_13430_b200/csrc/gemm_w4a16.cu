@@ -262,13 +262,15 @@ struct SmemPlan {
   static constexpr int kXTileBytes = TOK * kBlockK * 2;
   // int4 path: A stage = 4 KiB of packed nibbles; bf16 path: A stage = 16 KiB bf16 tile (read by the MMA)
   static constexpr int kAStageBytes = DEQUANT ? kPackedTileBytes : kWTileBytes;
-  static constexpr int kAStages = DEQUANT ? cmin(6, (512 - kAccCols) / kATmemColsPerStage) : 4;
   static constexpr int kPassTok = TOK < 64 ? TOK : 64;
   static constexpr int kPasses = TOK / kPassTok;
   static constexpr int kStagingBufBytes = kPassTok * kTileN * 2;
   static constexpr int kStagingBytes = OUT_MODE == kOutBf16 ? 2 * kStagingBufBytes : 0;
-  static constexpr int kFixedBytes = kAStages * kAStageBytes + kStagingBytes + kScaleSlots * kCookedScaleBytes + 1024 + 1024;
-  static constexpr int kBStages = DEQUANT ? cmin(8, (kSmemBudget - kFixedBytes) / kXTileBytes) : kAStages;
+  static constexpr int kFixedBytes = kStagingBytes + kScaleSlots * kCookedScaleBytes + 1024 + 1024;
+  // both rings have the same depth: one tcgen05.commit per k-block releases a stage of each
+  static constexpr int kStagesTmem = DEQUANT ? (512 - kAccCols) / kATmemColsPerStage : 8;
+  static constexpr int kAStages = cmin(cmin(8, kStagesTmem), (kSmemBudget - kFixedBytes) / (kXTileBytes + kAStageBytes));
+  static constexpr int kBStages = kAStages;
   static_assert(kBStages >= 2 && kAStages >= 2, "pipelines need at least two stages");
   static constexpr int kOffB = 0;
   static constexpr int kOffA = kBStages * kXTileBytes;
@@ -361,7 +363,9 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     *never_set = 0;
     *epi_stop = 0x7fffffff;
     for (int s = 0; s < kBStages; ++s) {
-      mbar_init(bar_b_full(s), 1);
+      // one barrier tells the MMA warp that a stage is ready: the activation tile has landed and
+      // (int4 path) the eight de-quantiser warps have written the A stage, or (bf16 path) the weight tile has landed
+      mbar_init(bar_b_full(s), DEQUANT ? 1 + kNumDeqWarps : 2);
       mbar_init(bar_b_empty(s), 1);
     }
     for (int s = 0; s < kAStages; ++s) {
@@ -403,14 +407,16 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             mbar_arrive_expect_tx(bar_b_full(ring.s), Plan::kXTileBytes);
             tma_load_2d(base + Plan::kOffB + ring.s * Plan::kXTileBytes, &tmap_x, bar_b_full(ring.s), kb * kBlockK, w.tok0);
           } else {
-            if (!mbar_wait(bar_a_empty(ring.s), ring.ph ^ 1u, abort_flag)) { ok = false; break; }
-            mbar_arrive_expect_tx(bar_a_full(ring.s), Plan::kAStageBytes);
+            if (!mbar_wait(bar_b_empty(ring.s), ring.ph ^ 1u, abort_flag)) { ok = false; break; }
             const uint32_t dst = base + Plan::kOffA + ring.s * Plan::kAStageBytes;
-            if (DEQUANT)
+            if (DEQUANT) {
+              mbar_arrive_expect_tx(bar_a_full(ring.s), Plan::kAStageBytes);
               bulk_load(dst, L.wq + ((size_t)(w.n0 / kTileN) * p.num_kb + kb) * kPackedTileBytes, kPackedTileBytes,
                         bar_a_full(ring.s));
-            else
-              tma_load_2d(dst, &tmap_w, bar_a_full(ring.s), kb * kBlockK, w.n0);
+            } else {
+              mbar_arrive_expect_tx(bar_b_full(ring.s), Plan::kAStageBytes);
+              tma_load_2d(dst, &tmap_w, bar_b_full(ring.s), kb * kBlockK, w.n0);
+            }
           }
           ring.next(stages);
           ++issued;
@@ -422,7 +428,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         const int pending = min(issued, stages);
         for (int j = 0; j < pending; ++j) {
           const int idx = issued - 1 - j;
-          const uint32_t bar = is_b ? bar_b_full(idx % stages) : bar_a_full(idx % stages);
+          const uint32_t bar = (is_b || !DEQUANT) ? bar_b_full(idx % stages) : bar_a_full(idx % stages);
           mbar_wait(bar, (uint32_t)(idx / stages) & 1u, never_set);
         }
       }
@@ -439,7 +445,6 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         if (!mbar_wait(bar_acc_empty, ((uint32_t)useq & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         tcgen05_fence_after();
         for (int it = 0; it < w.nkb; ++it) {
-          if (!mbar_wait(DEQUANT ? bar_a_deq(ra.s) : bar_a_full(ra.s), ra.ph, abort_flag)) { ok = false; break; }
           if (!mbar_wait(bar_b_full(rb.s), rb.ph, abort_flag)) { ok = false; break; }
           tcgen05_fence_after();
           const uint64_t bdesc = umma_desc_k_major_sw128(base + Plan::kOffB + rb.s * Plan::kXTileBytes);
@@ -456,8 +461,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
               umma_bf16(tmem_d, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
                         (it > 0 || k > 0) ? 1u : 0u);
           }
-          umma_commit(bar_a_empty(ra.s));
-          umma_commit(bar_b_empty(rb.s));
+          umma_commit(bar_b_empty(rb.s));                 // releases stage s of both rings
           ra.next(kAStages);
           rb.next(kBStages);
         }
@@ -561,7 +565,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                         (uint32_t)(ra.s * kATmemColsPerStage + h * 16), outw);
           tcgen05_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(bar_a_deq(ra.s));
+          if (lane == 0) mbar_arrive(bar_b_full(ra.s));
           ra.next(kAStages);
         }
       }
