@@ -177,6 +177,17 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
       : "memory");
 }
+// One lane of the (converged) warp; the surrounding code stays warp-uniform, so that loop state
+// and descriptors live in uniform registers.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ void tcgen05_fence_before() {
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
 }
@@ -435,19 +446,21 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16(kTileN, TOK);
-      Ring ra, rb;
-      int useq = 0;
-      for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x, ++useq) {
-        const Unit w = decode_unit(p, u, TOK);
-        // the epilogue warps must have drained the previous unit's accumulator
-        if (!mbar_wait(bar_acc_empty, ((uint32_t)useq & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+    // The whole warp walks the loop (warp-uniform control flow and addresses); one elected lane
+    // issues the MMAs and the commits.
+    constexpr uint32_t idesc = umma_idesc_bf16(kTileN, TOK);
+    Ring ra, rb;
+    int useq = 0;
+    for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x, ++useq) {
+      const Unit w = decode_unit(p, u, TOK);
+      // the epilogue warps must have drained the previous unit's accumulator
+      if (!mbar_wait(bar_acc_empty, ((uint32_t)useq & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+      tcgen05_fence_after();
+      for (int it = 0; it < w.nkb; ++it) {
+        if (!mbar_wait(bar_b_full(rb.s), rb.ph, abort_flag)) { ok = false; break; }
         tcgen05_fence_after();
-        for (int it = 0; it < w.nkb; ++it) {
-          if (!mbar_wait(bar_b_full(rb.s), rb.ph, abort_flag)) { ok = false; break; }
-          tcgen05_fence_after();
-          const uint64_t bdesc = umma_desc_k_major_sw128(base + Plan::kOffB + rb.s * Plan::kXTileBytes);
+        const uint64_t bdesc = umma_desc_k_major_sw128(base + Plan::kOffB + rb.s * Plan::kXTileBytes);
+        if (elect_one()) {
           if (DEQUANT) {
             const uint32_t a_tmem = tmem_d + kAccCols + (uint32_t)(ra.s * kATmemColsPerStage);
 #pragma unroll
@@ -462,13 +475,15 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                         (it > 0 || k > 0) ? 1u : 0u);
           }
           umma_commit(bar_b_empty(rb.s));                 // releases stage s of both rings
-          ra.next(kAStages);
-          rb.next(kBStages);
         }
-        if (ok) umma_commit(bar_acc_full);
+        __syncwarp();
+        ra.next(kAStages);
+        rb.next(kBStages);
       }
-      if (!ok) *abort_flag = 1;
+      if (ok && elect_one()) umma_commit(bar_acc_full);
+      __syncwarp();
     }
+    if (!ok) *abort_flag = 1;
   } else if (warp < kFirstDeqWarp) {
     // ------------------------------------------------------------------ scale warps
     if (DEQUANT) {
