@@ -188,9 +188,8 @@ __global__ void rope_kernel(__nv_bfloat16* __restrict__ q, __nv_bfloat16* __rest
 }
 
 // Causal attention with online softmax on the legacy tensor-core path (mma.sync m16n8k16,
-// bf16 in, fp32 accumulate).  One CTA = 64 queries of one (batch, head); each of the four
-// warps owns 16 query rows; keys are walked in blocks of 64 up to the diagonal block.
-// Attention is ~0.5 % of a step's FLOPs, so it stays off the tcgen05 path.
+// bf16 in, fp32 accumulate).  Attention is ~0.5 % of a step's FLOPs, so it stays off the
+// tcgen05 path.
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
@@ -209,125 +208,149 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// 16-byte asynchronous copy global -> shared; bytes = 0 fills the destination with zeros.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// One CTA = 128 queries of one (batch, head), eight warps of 16 query rows each; keys are walked in
+// blocks of 64 up to the diagonal, K and V blocks double-buffered with cp.async.  Query blocks are
+// scheduled from the last (most key blocks) to the first.
+constexpr int kAttBQ = 128, kAttBK = 64, kAttThreads = 256;
+
 template <int DH>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(kAttThreads, 2)
 attention_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                      const __nv_bfloat16* __restrict__ v, int ldq, int ldk, int ldv,
                      __nv_bfloat16* __restrict__ out, int ldo, int S, float scale_log2e) {
-  constexpr int BQ = 64, BK = 64;
+  constexpr int BQ = kAttBQ, BK = kAttBK;
   constexpr int LD = DH + 8;                       // padded row (bf16 elements): conflict-free ldmatrix
+  constexpr int CH = DH / 8;                       // 16-byte chunks per row
   extern __shared__ __align__(16) uint8_t att_smem[];
   __nv_bfloat16* sQ = reinterpret_cast<__nv_bfloat16*>(att_smem);
-  __nv_bfloat16* sK = sQ + BQ * LD;
-  __nv_bfloat16* sV = sK + BK * LD;
+  __nv_bfloat16* sKV = sQ + BQ * LD;               // [2 buffers][K | V][BK][LD]
 
-  const int qb = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int qb = (int)gridDim.x - 1 - (int)blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t4 = lane & 3;
   const size_t tok_base = (size_t)b * S;
   const int q0 = qb * BQ;
+  const int last_q = min(q0 + BQ, S) - 1;
+  const int nkb = last_q / BK + 1;                 // key blocks up to the diagonal of the last query row
 
-  // stage a [64][DH] tile (rows beyond S are zero)
-  auto load_tile = [&](__nv_bfloat16* dst, const __nv_bfloat16* src, int ld, int row0) {
-    constexpr int CH = DH / 8;                     // 16-byte chunks per row
-    for (int i = threadIdx.x; i < 64 * CH; i += 128) {
+  auto load_rows = [&](__nv_bfloat16* dst, const __nv_bfloat16* src, int ld, int row0, int rows) {
+    for (int i = threadIdx.x; i < rows * CH; i += kAttThreads) {
       const int r = i / CH, c = i % CH;
-      uint4 val = make_uint4(0, 0, 0, 0);
-      if (row0 + r < S) val = *reinterpret_cast<const uint4*>(src + (tok_base + row0 + r) * ld + h * DH + c * 8);
-      *reinterpret_cast<uint4*>(dst + r * LD + c * 8) = val;
+      const bool in = row0 + r < S;
+      const __nv_bfloat16* gp = src + (tok_base + (in ? row0 + r : 0)) * ld + h * DH + c * 8;
+      cp_async16((uint32_t)__cvta_generic_to_shared(dst + r * LD + c * 8), gp, in ? 16 : 0);
     }
   };
-  load_tile(sQ, q, ldq, q0);
+  auto load_kv = [&](int buf, int kb) {
+    __nv_bfloat16* dk = sKV + (size_t)buf * 2 * BK * LD;
+    load_rows(dk, k, ldk, kb * BK, BK);
+    load_rows(dk + BK * LD, v, ldv, kb * BK, BK);
+  };
+  load_rows(sQ, q, ldq, q0, BQ);
+  load_kv(0, 0);
+  cp_async_commit();
+  if (nkb > 1) load_kv(1, 1);
+  cp_async_commit();
+  cp_async_wait<1>();                              // Q and the first K/V block have landed
   __syncthreads();
 
-  // Q fragments of this warp's 16 rows, all of DH
-  uint32_t qf[DH / 16][4];
-  {
-    const int row = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-#pragma unroll
-    for (int kk = 0; kk < DH / 16; ++kk) {
-      const int col = kk * 16 + (lane >> 4) * 8;
-      ldmatrix_x4((uint32_t)__cvta_generic_to_shared(sQ + row * LD + col), qf[kk][0], qf[kk][1], qf[kk][2], qf[kk][3]);
-    }
-  }
+  // the Q fragments of this warp's 16 rows are re-read from shared memory in every key block
+  // (keeping them in registers would cost a second resident CTA per SM)
+  const int qfrag_row = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
   float o[DH / 8][4];
 #pragma unroll
   for (int i = 0; i < DH / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.0f;
   float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.0f, l1 = 0.0f;      // rows g and g + 8 of the warp's 16
   const int qrow0 = q0 + warp * 16 + g, qrow1 = qrow0 + 8;
+  const int warp_last_q = q0 + warp * 16 + 15;
 
-  for (int kb = 0; kb <= qb; ++kb) {
-    __syncthreads();                                // previous K/V tiles fully consumed
-    load_tile(sK, k, ldk, kb * BK);
-    load_tile(sV, v, ldv, kb * BK);
-    __syncthreads();
-
-    // scores: 16 x 64 per warp
-    float sc[BK / 8][4];
+  for (int kb = 0; kb < nkb; ++kb) {
+    const __nv_bfloat16* sK = sKV + (size_t)(kb & 1) * 2 * BK * LD;
+    const __nv_bfloat16* sV = sK + BK * LD;
+    if (kb * BK <= warp_last_q) {                   // warp-uniform: this key block reaches the warp's rows
+      // scores: 16 x 64 per warp
+      float sc[BK / 8][4];
 #pragma unroll
-    for (int j = 0; j < BK / 8; ++j) sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.0f;
+      for (int j = 0; j < BK / 8; ++j) sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.0f;
 #pragma unroll
-    for (int kk = 0; kk < DH / 16; ++kk) {
+      for (int kk = 0; kk < DH / 16; ++kk) {
+        uint32_t qf[4];
+        ldmatrix_x4((uint32_t)__cvta_generic_to_shared(sQ + qfrag_row * LD + kk * 16 + (lane >> 4) * 8),
+                    qf[0], qf[1], qf[2], qf[3]);
 #pragma unroll
-      for (int jp = 0; jp < BK / 16; ++jp) {        // two n8 tiles (16 keys) per ldmatrix.x4
-        uint32_t b00, b01, b10, b11;
-        const int key = jp * 16 + (lane & 7) + (lane >> 4) * 8;
-        const int col = kk * 16 + ((lane >> 3) & 1) * 8;
-        ldmatrix_x4((uint32_t)__cvta_generic_to_shared(sK + key * LD + col), b00, b01, b10, b11);
-        mma_bf16_16816(sc[2 * jp], qf[kk], b00, b01);
-        mma_bf16_16816(sc[2 * jp + 1], qf[kk], b10, b11);
+        for (int jp = 0; jp < BK / 16; ++jp) {      // two n8 tiles (16 keys) per ldmatrix.x4
+          uint32_t b00, b01, b10, b11;
+          const int key = jp * 16 + (lane & 7) + (lane >> 4) * 8;
+          const int col = kk * 16 + ((lane >> 3) & 1) * 8;
+          ldmatrix_x4((uint32_t)__cvta_generic_to_shared(sK + key * LD + col), b00, b01, b10, b11);
+          mma_bf16_16816(sc[2 * jp], qf, b00, b01);
+          mma_bf16_16816(sc[2 * jp + 1], qf, b10, b11);
+        }
       }
-    }
-    // causal mask (only the diagonal block can cross it)
-    if (kb == qb) {
+      // causal mask (only blocks that reach past the warp's first row can cross it)
+      if (kb * BK + BK - 1 > q0 + warp * 16) {
+#pragma unroll
+        for (int j = 0; j < BK / 8; ++j) {
+          const int key = kb * BK + j * 8 + 2 * t4;
+          if (key > qrow0) sc[j][0] = -INFINITY;
+          if (key + 1 > qrow0) sc[j][1] = -INFINITY;
+          if (key > qrow1) sc[j][2] = -INFINITY;
+          if (key + 1 > qrow1) sc[j][3] = -INFINITY;
+        }
+      }
+      // online softmax (base-2 exponent with the 1/sqrt(dh) scale folded in)
+      float mx0 = m0, mx1 = m1;
 #pragma unroll
       for (int j = 0; j < BK / 8; ++j) {
-        const int key = kb * BK + j * 8 + 2 * t4;
-        if (key > qrow0) sc[j][0] = -INFINITY;
-        if (key + 1 > qrow0) sc[j][1] = -INFINITY;
-        if (key > qrow1) sc[j][2] = -INFINITY;
-        if (key + 1 > qrow1) sc[j][3] = -INFINITY;
+        mx0 = fmaxf(mx0, fmaxf(sc[j][0], sc[j][1]));
+        mx1 = fmaxf(mx1, fmaxf(sc[j][2], sc[j][3]));
+      }
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+      const float corr0 = exp2f((m0 - mx0) * scale_log2e), corr1 = exp2f((m1 - mx1) * scale_log2e);
+      m0 = mx0; m1 = mx1;
+      float rs0 = 0.0f, rs1 = 0.0f;
+      uint32_t pf[BK / 16][4];
+#pragma unroll
+      for (int j = 0; j < BK / 8; ++j) {
+        const float p0 = exp2f((sc[j][0] - mx0) * scale_log2e), p1 = exp2f((sc[j][1] - mx0) * scale_log2e);
+        const float p2 = exp2f((sc[j][2] - mx1) * scale_log2e), p3 = exp2f((sc[j][3] - mx1) * scale_log2e);
+        rs0 += p0 + p1; rs1 += p2 + p3;
+        pf[j >> 1][(j & 1) * 2] = pack_bf16x2(p0, p1);
+        pf[j >> 1][(j & 1) * 2 + 1] = pack_bf16x2(p2, p3);
+      }
+      l0 = l0 * corr0 + rs0; l1 = l1 * corr1 + rs1;
+#pragma unroll
+      for (int i = 0; i < DH / 8; ++i) { o[i][0] *= corr0; o[i][1] *= corr0; o[i][2] *= corr1; o[i][3] *= corr1; }
+      // O += P V
+#pragma unroll
+      for (int kk = 0; kk < BK / 16; ++kk) {
+#pragma unroll
+        for (int np = 0; np < DH / 16; ++np) {      // two n8 tiles of the head dimension per ldmatrix.x4.trans
+          uint32_t b00, b01, b10, b11;
+          const int key = kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+          const int col = np * 16 + (lane >> 4) * 8;
+          ldmatrix_x4_trans((uint32_t)__cvta_generic_to_shared(sV + key * LD + col), b00, b01, b10, b11);
+          mma_bf16_16816(o[2 * np], pf[kk], b00, b01);
+          mma_bf16_16816(o[2 * np + 1], pf[kk], b10, b11);
+        }
       }
     }
-    // online softmax (base-2 exponent with the 1/sqrt(dh) scale folded in)
-    float mx0 = m0, mx1 = m1;
-#pragma unroll
-    for (int j = 0; j < BK / 8; ++j) {
-      mx0 = fmaxf(mx0, fmaxf(sc[j][0], sc[j][1]));
-      mx1 = fmaxf(mx1, fmaxf(sc[j][2], sc[j][3]));
-    }
-    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-    const float corr0 = exp2f((m0 - mx0) * scale_log2e), corr1 = exp2f((m1 - mx1) * scale_log2e);
-    m0 = mx0; m1 = mx1;
-    float rs0 = 0.0f, rs1 = 0.0f;
-    uint32_t pf[BK / 16][4];
-#pragma unroll
-    for (int j = 0; j < BK / 8; ++j) {
-      const float p0 = exp2f((sc[j][0] - mx0) * scale_log2e), p1 = exp2f((sc[j][1] - mx0) * scale_log2e);
-      const float p2 = exp2f((sc[j][2] - mx1) * scale_log2e), p3 = exp2f((sc[j][3] - mx1) * scale_log2e);
-      rs0 += p0 + p1; rs1 += p2 + p3;
-      pf[j >> 1][(j & 1) * 2] = pack_bf16x2(p0, p1);
-      pf[j >> 1][(j & 1) * 2 + 1] = pack_bf16x2(p2, p3);
-    }
-    l0 = l0 * corr0 + rs0; l1 = l1 * corr1 + rs1;
-#pragma unroll
-    for (int i = 0; i < DH / 8; ++i) { o[i][0] *= corr0; o[i][1] *= corr0; o[i][2] *= corr1; o[i][3] *= corr1; }
-    // O += P V
-#pragma unroll
-    for (int kk = 0; kk < BK / 16; ++kk) {
-#pragma unroll
-      for (int np = 0; np < DH / 16; ++np) {        // two n8 tiles of the head dimension per ldmatrix.x4.trans
-        uint32_t b00, b01, b10, b11;
-        const int key = kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-        const int col = np * 16 + (lane >> 4) * 8;
-        ldmatrix_x4_trans((uint32_t)__cvta_generic_to_shared(sV + key * LD + col), b00, b01, b10, b11);
-        mma_bf16_16816(o[2 * np], pf[kk], b00, b01);
-        mma_bf16_16816(o[2 * np + 1], pf[kk], b10, b11);
-      }
-    }
+    __syncthreads();                                // every warp is done with buffer kb & 1
+    if (kb + 2 < nkb) load_kv(kb & 1, kb + 2);
+    cp_async_commit();
+    cp_async_wait<1>();                             // block kb + 1 has landed (for this thread's copies)
+    __syncthreads();
   }
   // normalise and store
   l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
@@ -452,18 +475,18 @@ int launch_rope(__nv_bfloat16* q, __nv_bfloat16* k, int ldq, int ldk, const floa
 int launch_attention(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v, int ldq, int ldk, int ldv,
                      __nv_bfloat16* out, int ldo, int B, int S, int H, int dh, cudaStream_t st) {
   const float scale_log2e = 1.4426950408889634f / sqrtf((float)dh);
-  const dim3 grid(ceil_div(S, 64), H, B);
+  const dim3 grid(ceil_div(S, kAttBQ), H, B);
   if ((ldq % 8) || (ldk % 8) || (ldv % 8) || (ldo % 2)) return QZO_ERR_BAD_ARG;
   if (dh == 64) {
-    constexpr int smem = 3 * 64 * (64 + 8) * 2;
+    constexpr int smem = (kAttBQ + 4 * kAttBK) * (64 + 8) * 2;
     static bool cfg = false;
     if (!cfg) { QZO_CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)); cfg = true; }
-    QZO_LAUNCH(attention_mma_kernel<64>, grid, dim3(128), smem, st, q, k, v, ldq, ldk, ldv, out, ldo, S, scale_log2e);
+    QZO_LAUNCH(attention_mma_kernel<64>, grid, dim3(kAttThreads), smem, st, q, k, v, ldq, ldk, ldv, out, ldo, S, scale_log2e);
   } else if (dh == 128) {
-    constexpr int smem = 3 * 64 * (128 + 8) * 2;
+    constexpr int smem = (kAttBQ + 4 * kAttBK) * (128 + 8) * 2;
     static bool cfg = false;
     if (!cfg) { QZO_CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)); cfg = true; }
-    QZO_LAUNCH(attention_mma_kernel<128>, grid, dim3(128), smem, st, q, k, v, ldq, ldk, ldv, out, ldo, S, scale_log2e);
+    QZO_LAUNCH(attention_mma_kernel<128>, grid, dim3(kAttThreads), smem, st, q, k, v, ldq, ldk, ldv, out, ldo, S, scale_log2e);
   } else {
     return QZO_ERR_BAD_ARG;
   }
