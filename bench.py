@@ -19,6 +19,10 @@ import time
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
+# dram__bytes_read.sum + dram__bytes_write.sum over algorithmic bytes of the captured GEMM launch;
+# set to None whenever the GEMM kernel changes after the capture.
+NCU_TRAFFIC_RATIO = (57.42e6 + 55.72e6) / 146.98e6
+
 
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -234,6 +238,16 @@ def main():
             dist.destroy_process_group()
         return
 
+    # DRAM traffic of the dominant kernel: measured once with ncu on the 4096 x 11008, M = 4096 sweep
+    # launch (profiles/w4a16_gemm_K4096_N11008_M4096.txt: 57.4 MB read + 55.7 MB written for 147.0 MB
+    # of algorithmic bytes) and scaled to this step's mean launch by algorithmic bytes.
+    def gemm_bytes(M, K, N):
+        return K * N // 2 + 2 * ((K + 127) // 128) * N + 2 * M * K + 2 * M * N
+    shapes = inputs.linear_shapes(cfg)
+    T = B * S
+    launches_per_layer = 4 if cfg["arch"] == "llama" else 4          # qkv, o, (gate+up | fc1), (down | fc2)
+    mean_bytes = sum(gemm_bytes(T, K, N) for _, K, N in shapes) / launches_per_layer
+    traffic = NCU_TRAFFIC_RATIO * mean_bytes if NCU_TRAFFIC_RATIO else None
     peaks = measured_peaks()
     value = replicas.whole_job_rate(args.steps, world, ms)
     e2e = replicas.whole_job_rate(args.steps, world, e2e_ms)
@@ -247,7 +261,8 @@ def main():
             "gpu_launches": int(launches),
             "roofline": {"kernel": "w4a16_gemm_kernel (perturbed W4A16 GEMM, all block linears)", "bound": "tensor",
                          "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-                         "peak_source": f"{peaks['source']} bf16 sustained", "traffic": None,
+                         "peak_source": f"{peaks['source']} bf16 sustained", "traffic": traffic, "traffic_unit": "bytes per launch (ncu, scaled from the sweep launch)",
+                         "algorithmic_bytes_per_launch": mean_bytes,
                          "launches": int(n_l), "gemm_share_of_step": gemm_ms / ms if ms > 0 else None}}
     if not args.no_cpu_baseline:
         v, cores, desc = oracle_sample(workload, n_seq=8)
