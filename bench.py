@@ -212,6 +212,8 @@ def main():
     seed0 = 42
     for t in range(args.warmup):
         model.qzo_step(tok_d, lab_d, seed0 + t, c["eps"], c["lr"], c["clip"], read_back=False)
+        if t == 0 and model.qzo_device_status() != 0:
+            raise SystemExit("device status word set in the first step: a bounded wait expired")
     model.qzo_profile_gemms(n_gemm * args.steps)
     sampler = ClockSampler(local)
     if rank == 0:

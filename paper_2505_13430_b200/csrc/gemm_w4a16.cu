@@ -273,15 +273,16 @@ struct SmemPlan {
   static constexpr int kXTileBytes = TOK * kBlockK * 2;
   // int4 path: A stage = 4 KiB of packed nibbles; bf16 path: A stage = 16 KiB bf16 tile (read by the MMA)
   static constexpr int kAStageBytes = DEQUANT ? kPackedTileBytes : kWTileBytes;
-  static constexpr int kPassTok = TOK < 64 ? TOK : 64;
+  static constexpr int kPassTok = TOK < 32 ? TOK : 32;
   static constexpr int kPasses = TOK / kPassTok;
   static constexpr int kStagingBufBytes = kPassTok * kTileN * 2;
   static constexpr int kStagingBytes = OUT_MODE == kOutBf16 ? 2 * kStagingBufBytes : 0;
   static constexpr int kFixedBytes = kStagingBytes + kScaleSlots * kCookedScaleBytes + 1024 + 1024;
-  // both rings have the same depth: one tcgen05.commit per k-block releases a stage of each
-  static constexpr int kStagesTmem = DEQUANT ? (512 - kAccCols) / kATmemColsPerStage : 8;
-  static constexpr int kAStages = cmin(cmin(8, kStagesTmem), (kSmemBudget - kFixedBytes) / (kXTileBytes + kAStageBytes));
-  static constexpr int kBStages = kAStages;
+  // int4 path: the A ring (4 KiB of nibbles + 32 TMEM columns per stage) is as deep as tensor memory
+  // allows, the B ring takes the shared memory that is left; bf16 path: both rings alike
+  static constexpr int kStagesTmem = (512 - kAccCols) / kATmemColsPerStage;
+  static constexpr int kAStages = DEQUANT ? cmin(8, kStagesTmem) : 4;
+  static constexpr int kBStages = DEQUANT ? cmin(8, (kSmemBudget - kFixedBytes - kAStages * kAStageBytes) / kXTileBytes) : 4;
   static_assert(kBStages >= 2 && kAStages >= 2, "pipelines need at least two stages");
   static constexpr int kOffB = 0;
   static constexpr int kOffA = kBStages * kXTileBytes;
@@ -374,9 +375,10 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     *never_set = 0;
     *epi_stop = 0x7fffffff;
     for (int s = 0; s < kBStages; ++s) {
-      // one barrier tells the MMA warp that a stage is ready: the activation tile has landed and
-      // (int4 path) the eight de-quantiser warps have written the A stage, or (bf16 path) the weight tile has landed
-      mbar_init(bar_b_full(s), DEQUANT ? 1 + kNumDeqWarps : 2);
+      // bf16 path: one barrier tells the MMA warp that both tiles of a stage have landed (rings of
+      // equal depth).  int4 path: the A ring is deeper than the B ring, so the de-quantisers signal
+      // their own barrier (an arrival on the B barrier could fall into its previous phase)
+      mbar_init(bar_b_full(s), DEQUANT ? 1 : 2);
       mbar_init(bar_b_empty(s), 1);
     }
     for (int s = 0; s < kAStages; ++s) {
@@ -418,7 +420,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             mbar_arrive_expect_tx(bar_b_full(ring.s), Plan::kXTileBytes);
             tma_load_2d(base + Plan::kOffB + ring.s * Plan::kXTileBytes, &tmap_x, bar_b_full(ring.s), kb * kBlockK, w.tok0);
           } else {
-            if (!mbar_wait(bar_b_empty(ring.s), ring.ph ^ 1u, abort_flag)) { ok = false; break; }
+            if (!mbar_wait(bar_a_empty(ring.s), ring.ph ^ 1u, abort_flag)) { ok = false; break; }
             const uint32_t dst = base + Plan::kOffA + ring.s * Plan::kAStageBytes;
             if (DEQUANT) {
               mbar_arrive_expect_tx(bar_a_full(ring.s), Plan::kAStageBytes);
@@ -457,6 +459,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
       if (!mbar_wait(bar_acc_empty, ((uint32_t)useq & 1u) ^ 1u, abort_flag)) { ok = false; break; }
       tcgen05_fence_after();
       for (int it = 0; it < w.nkb; ++it) {
+        if (DEQUANT && !mbar_wait(bar_a_deq(ra.s), ra.ph, abort_flag)) { ok = false; break; }
         if (!mbar_wait(bar_b_full(rb.s), rb.ph, abort_flag)) { ok = false; break; }
         tcgen05_fence_after();
         const uint64_t bdesc = umma_desc_k_major_sw128(base + Plan::kOffB + rb.s * Plan::kXTileBytes);
@@ -474,7 +477,8 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
               umma_bf16(tmem_d, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
                         (it > 0 || k > 0) ? 1u : 0u);
           }
-          umma_commit(bar_b_empty(rb.s));                 // releases stage s of both rings
+          umma_commit(bar_b_empty(rb.s));                 // releases the stage of each ring
+          umma_commit(bar_a_empty(ra.s));
         }
         __syncwarp();
         ra.next(kAStages);
@@ -580,7 +584,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                         (uint32_t)(ra.s * kATmemColsPerStage + h * 16), outw);
           tcgen05_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(bar_b_full(ra.s));
+          if (lane == 0) mbar_arrive(bar_a_deq(ra.s));
           ra.next(kAStages);
         }
       }
@@ -830,7 +834,7 @@ int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const Ge
   if (splits <= 1) {
     for (int j = 0; j < kMaxGroupedLinears; ++j) {
       const GemmLinear& g = lins[j < n_lin ? j : 0];
-      QZO_TRY(make_tmap_bf16(&ty[j], g.out, M, g.N, g.ldo, kTileN, tok < 64 ? tok : 64, false));
+      QZO_TRY(make_tmap_bf16(&ty[j], g.out, M, g.N, g.ldo, kTileN, tok < 32 ? tok : 32, false));
     }
     p.splits = 1;
     p.kb_per_split = ceil_div(p.num_kb, 2) * 2;
