@@ -3,9 +3,9 @@
 * The standalone perturbed W4A16 GEMM on every K x N and token count of the sweep, in the launch
   configuration the sweep times (same entry point, same tile / split-K choice): sampled rows and
   columns (first and last tile, ragged edges, random ones) against the oracle, max relative 2e-2.
-* One full-width decoder block of the Llama-2-7B shape at the benchmark's batch (16 x 256 tokens,
-  so the grouped q/k/v and gate/up launches and the 256-token tiles are the ones the benchmark
-  runs): block output and logits of sampled sequences against the oracle (sequences of a batch do
+* One full-width decoder block of the Llama-2-7B shape (16 x 256 tokens) and of the OPT-6.7B shape
+  (32 x 128 tokens; LayerNorm, biases, ReLU, learned positions) at the benchmark's batch, so the
+  grouped q/k/v and gate/up launches and the 256-token tiles are the ones the benchmark runs: block output and logits of sampled sequences against the oracle (sequences of a batch do
   not interact, so the oracle needs only those sequences).
 """
 import numpy as np
@@ -60,14 +60,15 @@ def test_sweep_shapes_match_oracle_on_sampled_outputs(lib, M, K, N):
         assert bool(torch.isfinite(y.float()).all())
 
 
-def test_full_width_llama7b_block_matches_oracle_on_sampled_sequences(lib):
-    c = inputs.CONFIGS["llama7b"]
-    cfg = inputs.model_cfg("llama7b", n_layers=1)
+@pytest.mark.parametrize("workload", ["llama7b", "opt6.7b"])
+def test_full_width_block_matches_oracle_on_sampled_sequences(lib, workload):
+    c = inputs.CONFIGS[workload]
+    cfg = inputs.model_cfg(workload, n_layers=1)
     raw = inputs.raw_model_tensors(cfg, seed=1000)
     om = build_oracle_model(raw)
     quant = {(0, name): (torch.from_numpy(int4.pack_int4(om["layers"][0]["lin"][name]["q"]).view(np.int32)),
                          torch.from_numpy(om["layers"][0]["lin"][name]["s"]).bfloat16())
-             for name in omodel.LINEAR_ORDER["llama"]}
+             for name in omodel.LINEAR_ORDER[cfg["arch"]]}
     B, S = c["batch"], c["seq"]
     gm = lib.build_model_from_raw(raw, B * S, quantized=quant)
     del raw
