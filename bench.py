@@ -267,7 +267,7 @@ def main():
                          "algorithmic_bytes_per_launch": mean_bytes,
                          "launches": int(n_l), "gemm_share_of_step": gemm_ms / ms if ms > 0 else None}}
     if not args.no_cpu_baseline:
-        v, cores, desc = oracle_sample(workload, n_seq=8)
+        v, cores, desc = oracle_sample(workload, n_seq=16)
         line["cpu_baseline"] = {"value": v, "unit": "steps/s", "cores": cores, "kind": "oracle", "sample": desc}
     print(json.dumps(line))
     if world > 1:
