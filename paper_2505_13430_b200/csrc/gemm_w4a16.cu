@@ -227,8 +227,8 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t v[16]) 
       ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
         "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
       : "memory");
-  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -281,9 +281,13 @@ struct SmemPlan {
   // int4 path: the A ring (4 KiB of nibbles + 32 TMEM columns per stage) is as deep as tensor memory
   // allows, the B ring takes the shared memory that is left; bf16 path: both rings alike
   static constexpr int kStagesTmem = (512 - kAccCols) / kATmemColsPerStage;
-  static constexpr int kAStages = DEQUANT ? cmin(8, kStagesTmem) : 4;
+  // A slot of the int4 path = one quantisation group = two k-blocks: one 8 KiB bulk copy, one wait
+  // and one arrival per group for the producer, the de-quantisers and the MMA warp
+  static constexpr int kAGroup = DEQUANT ? 2 : 1;                  // k-blocks per A-ring slot
+  static constexpr int kAStages = DEQUANT ? cmin(8, kStagesTmem) / 2 * 2 : 4;
+  static constexpr int kASlots = kAStages / kAGroup;
   static constexpr int kBStages = DEQUANT ? cmin(8, (kSmemBudget - kFixedBytes - kAStages * kAStageBytes) / kXTileBytes) : 4;
-  static_assert(kBStages >= 2 && kAStages >= 2, "pipelines need at least two stages");
+  static_assert(kBStages >= 2 && kASlots >= 2, "pipelines need at least two stages");
   static constexpr int kOffB = 0;
   static constexpr int kOffA = kBStages * kXTileBytes;
   static constexpr int kOffStaging = kOffA + kAStages * kAStageBytes;
@@ -341,6 +345,8 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                   const __grid_constant__ CUtensorMap tmap_y2, const __grid_constant__ GemmParams p) {
   using Plan = SmemPlan<TOK, DEQUANT, OUT_MODE>;
   constexpr int kAStages = Plan::kAStages;
+  constexpr int kASlots = Plan::kASlots;
+  constexpr int kAGroup = Plan::kAGroup;
   constexpr int kBStages = Plan::kBStages;
   constexpr uint32_t kAccCols = Plan::kAccCols;
   constexpr uint32_t kTmemCols = Plan::kTmemCols;
@@ -381,7 +387,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
       mbar_init(bar_b_full(s), DEQUANT ? 1 : 2);
       mbar_init(bar_b_empty(s), 1);
     }
-    for (int s = 0; s < kAStages; ++s) {
+    for (int s = 0; s < kASlots; ++s) {
       mbar_init(bar_a_full(s), 1);
       mbar_init(bar_a_deq(s), kNumDeqWarps);
       mbar_init(bar_a_empty(s), 1);
@@ -407,32 +413,38 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     // warp 0 feeds the B ring (activation tiles), warp 2 the A ring (packed nibbles / bf16 weights)
     if (lane == 0) {
       const bool is_b = warp == 0;
-      const int stages = is_b ? kBStages : kAStages;
+      const int stages = is_b ? kBStages : kASlots;
       Ring ring;
       int issued = 0;
       for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x) {
         const Unit w = decode_unit(p, u, TOK);
         const LinearDesc& L = p.lin[w.lin];
-        for (int it = 0; it < w.nkb; ++it) {
-          const int kb = w.kb_begin + it;
-          if (is_b) {
+        if (is_b) {
+          for (int it = 0; it < w.nkb; ++it) {
             if (!mbar_wait(bar_b_empty(ring.s), ring.ph ^ 1u, abort_flag)) { ok = false; break; }
             mbar_arrive_expect_tx(bar_b_full(ring.s), Plan::kXTileBytes);
-            tma_load_2d(base + Plan::kOffB + ring.s * Plan::kXTileBytes, &tmap_x, bar_b_full(ring.s), kb * kBlockK, w.tok0);
-          } else {
+            tma_load_2d(base + Plan::kOffB + ring.s * Plan::kXTileBytes, &tmap_x, bar_b_full(ring.s),
+                        (w.kb_begin + it) * kBlockK, w.tok0);
+            ring.next(stages);
+            ++issued;
+          }
+        } else {
+          for (int it = 0; it < w.nkb; it += kAGroup) {
+            const int kb = w.kb_begin + it;
+            const int nk = min(kAGroup, w.nkb - it);         // k-blocks of this slot (the last group of an odd K has one)
             if (!mbar_wait(bar_a_empty(ring.s), ring.ph ^ 1u, abort_flag)) { ok = false; break; }
-            const uint32_t dst = base + Plan::kOffA + ring.s * Plan::kAStageBytes;
+            const uint32_t dst = base + Plan::kOffA + ring.s * (kAGroup * Plan::kAStageBytes);
             if (DEQUANT) {
-              mbar_arrive_expect_tx(bar_a_full(ring.s), Plan::kAStageBytes);
-              bulk_load(dst, L.wq + ((size_t)(w.n0 / kTileN) * p.num_kb + kb) * kPackedTileBytes, kPackedTileBytes,
-                        bar_a_full(ring.s));
+              mbar_arrive_expect_tx(bar_a_full(ring.s), (uint32_t)(nk * kPackedTileBytes));
+              bulk_load(dst, L.wq + ((size_t)(w.n0 / kTileN) * p.num_kb + kb) * kPackedTileBytes,
+                        (uint32_t)(nk * kPackedTileBytes), bar_a_full(ring.s));
             } else {
               mbar_arrive_expect_tx(bar_b_full(ring.s), Plan::kAStageBytes);
               tma_load_2d(dst, &tmap_w, bar_b_full(ring.s), kb * kBlockK, w.n0);
             }
+            ring.next(stages);
+            ++issued;
           }
-          ring.next(stages);
-          ++issued;
         }
       }
       if (!ok) {
@@ -459,13 +471,15 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
       if (!mbar_wait(bar_acc_empty, ((uint32_t)useq & 1u) ^ 1u, abort_flag)) { ok = false; break; }
       tcgen05_fence_after();
       for (int it = 0; it < w.nkb; ++it) {
-        if (DEQUANT && !mbar_wait(bar_a_deq(ra.s), ra.ph, abort_flag)) { ok = false; break; }
+        const int j = it % kAGroup;                           // position inside the A slot
+        if (DEQUANT && j == 0 && !mbar_wait(bar_a_deq(ra.s), ra.ph, abort_flag)) { ok = false; break; }
         if (!mbar_wait(bar_b_full(rb.s), rb.ph, abort_flag)) { ok = false; break; }
         tcgen05_fence_after();
+        const bool slot_done = j == kAGroup - 1 || it == w.nkb - 1;
         const uint64_t bdesc = umma_desc_k_major_sw128(base + Plan::kOffB + rb.s * Plan::kXTileBytes);
         if (elect_one()) {
           if (DEQUANT) {
-            const uint32_t a_tmem = tmem_d + kAccCols + (uint32_t)(ra.s * kATmemColsPerStage);
+            const uint32_t a_tmem = tmem_d + kAccCols + (uint32_t)((ra.s * kAGroup + j) * kATmemColsPerStage);
 #pragma unroll
             for (int k = 0; k < kBlockK / 16; ++k)      // 16 bf16 along K = 8 TMEM columns
               umma_bf16_tmem_a(tmem_d, a_tmem + (uint32_t)(k * 8), bdesc + (uint64_t)(k * 2), idesc,
@@ -477,11 +491,11 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
               umma_bf16(tmem_d, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
                         (it > 0 || k > 0) ? 1u : 0u);
           }
-          umma_commit(bar_b_empty(rb.s));                 // releases the stage of each ring
-          umma_commit(bar_a_empty(ra.s));
+          umma_commit(bar_b_empty(rb.s));                 // releases the B stage
+          if (slot_done) umma_commit(bar_a_empty(ra.s));  // and, after its last k-block, the A slot
         }
         __syncwarp();
-        ra.next(kAStages);
+        if (slot_done) ra.next(kASlots);
         rb.next(kBStages);
       }
       if (ok && elect_one()) umma_commit(bar_acc_full);
@@ -546,12 +560,29 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
       __nv_bfloat162 s_hi, s_lo;
       *reinterpret_cast<uint32_t*>(&s_hi) = 0u;
       *reinterpret_cast<uint32_t*>(&s_lo) = 0u;
-      Ring ra;
+      // nibbles of one 16-byte unit (32 consecutive k of this thread's row) -> 16 x bf16x2 (u - 8) * s'
+      auto dequant16 = [&](const uint4& pk, uint32_t (&outw)[16]) {
+        const uint32_t words[4] = {pk.x, pk.y, pk.z, pk.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+#pragma unroll
+          for (int pp = 0; pp < 4; ++pp) {
+            uint32_t x = ((words[i] >> (4 * pp)) & 0x000F000Fu) | 0x43004300u;     // bf16x2 {128 + u_lo, 128 + u_hi}
+            __nv_bfloat162 q2 = __hsub2(*reinterpret_cast<__nv_bfloat162*>(&x), magic_bias);   // exact u - 8
+            __nv_bfloat162 w2 = __hfma2(q2, s_hi, __hmul2(q2, s_lo));
+            outw[i * 4 + pp] = *reinterpret_cast<uint32_t*>(&w2);                  // k = 32 h + 2 j, 2 j + 1 in register j
+          }
+        }
+      };
+      // A stage in tensor memory: lane = row (this warp's quadrant), column = k / 2
+      const uint32_t a_lane_base = tmem_d + ((uint32_t)((warp & 3) * 32) << 16) + kAccCols + (uint32_t)(h * 16);
+      Ring ra;                              // A-ring slot = one quantisation group (two k-blocks)
       int gig = 0;
       for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x) {
         const Unit w = decode_unit(p, u, TOK);
-        for (int it = 0; it < w.nkb; ++it) {
-          if ((it & 1) == 0) {
+        for (int it = 0; it < w.nkb; it += 2) {
+          const bool two = it + 1 < w.nkb;                    // the last group of an odd K has one k-block
+          {
             const int slot = gig % kScaleSlots;
             const uint32_t gph = (uint32_t)(gig / kScaleSlots) & 1u;
             ++gig;
@@ -562,30 +593,25 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_sc_empty(slot));
           }
-          // bar_a_full completing implies the stage was released by the MMAs that last read it
+          // bar_a_full completing implies the slot was released by the MMAs that last read it
           if (!__all_sync(0xffffffffu, mbar_wait(bar_a_full(ra.s), ra.ph, abort_flag))) { ok = false; break; }
-          tcgen05_fence_after();                              // orders the MMAs' reads of this A stage before the store below
-          const uint8_t* stage = smem + Plan::kOffA + ra.s * Plan::kAStageBytes;
-          const uint4 pk = *reinterpret_cast<const uint4*>(stage + (h * kTileN + r) * 16);
-          const uint32_t words[4] = {pk.x, pk.y, pk.z, pk.w};
-          uint32_t outw[16];                                  // k = 32 h + 2 j, 2 j + 1 in register j
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-#pragma unroll
-            for (int pp = 0; pp < 4; ++pp) {
-              uint32_t x = ((words[i] >> (4 * pp)) & 0x000F000Fu) | 0x43004300u;     // bf16x2 {128 + u_lo, 128 + u_hi}
-              __nv_bfloat162 q2 = __hsub2(*reinterpret_cast<__nv_bfloat162*>(&x), magic_bias);   // exact u - 8
-              __nv_bfloat162 w2 = __hfma2(q2, s_hi, __hmul2(q2, s_lo));
-              outw[i * 4 + pp] = *reinterpret_cast<uint32_t*>(&w2);
-            }
+          const uint8_t* src = smem + Plan::kOffA + ra.s * (2 * Plan::kAStageBytes) + (h * kTileN + r) * 16;
+          const uint4 pk0 = *reinterpret_cast<const uint4*>(src);
+          uint4 pk1 = make_uint4(0, 0, 0, 0);
+          if (two) pk1 = *reinterpret_cast<const uint4*>(src + Plan::kAStageBytes);
+          tcgen05_fence_after();                              // orders the MMAs' reads of this slot before the stores below
+          uint32_t outw[16];
+          dequant16(pk0, outw);
+          tmem_st16(a_lane_base + (uint32_t)((ra.s * 2) * kATmemColsPerStage), outw);
+          if (two) {
+            dequant16(pk1, outw);
+            tmem_st16(a_lane_base + (uint32_t)((ra.s * 2 + 1) * kATmemColsPerStage), outw);
           }
-          // A tile of the stage in tensor memory: lane = row (this warp's quadrant), column = k / 2
-          tmem_st16(tmem_d + ((uint32_t)((warp & 3) * 32) << 16) + kAccCols +
-                        (uint32_t)(ra.s * kATmemColsPerStage + h * 16), outw);
+          tmem_wait_st();
           tcgen05_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(bar_a_deq(ra.s));
-          ra.next(kAStages);
+          ra.next(kASlots);
         }
       }
       if (!ok) *abort_flag = 1;
