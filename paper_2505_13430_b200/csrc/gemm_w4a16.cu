@@ -16,14 +16,14 @@
 // the activations (q, k, v or gate, up) are served by one launch; the logical scale index of a
 // scale never depends on that grouping.
 //
-// Warp roles (21 warps):
+// Warp roles (23 warps):
 //   warp 0       TMA producer of the B ring: activation tiles (2-D tensor map, 128-byte swizzle)
 //   warp 1       MMA issuer (one elected lane), owns the TMEM allocation
-//   warp 2       TMA producer of the A ring: packed int4 tiles (one 4 KiB bulk copy per k-block)
-//   warps 3-4    scale warps: Philox4x32-10 + Box-Muller, s' = s + sign eps z in fp32, split
-//                into bf16 hi + lo parts, written to a small shared-memory ring
-//   warps 5-12   de-quantisers: nibbles -> bf16 (u - 8) * s' written to the A stage in TMEM
-//   warps 13-20  epilogue: TMEM -> registers (+ bias) -> bf16 rows in shared memory -> TMA stores;
+//   warp 2       producer of the A ring: packed int4 tiles (one 8 KiB bulk copy per quantisation group)
+//   warps 3-6    scale warps: Philox4x32-10 + Box-Muller, s' = s + sign eps z in fp32, split
+//                into bf16 hi + lo parts, written next to the nibbles of the group's A slot
+//   warps 7-14   de-quantisers: nibbles -> bf16 (u - 8) * s' written to the A stages in TMEM
+//   warps 15-22  epilogue: TMEM -> registers (+ bias) -> bf16 rows in shared memory -> TMA stores;
 //                runs while the other warps already work on the next unit
 // Every wait on an mbarrier is bounded; when a wait expires the CTA records an error in
 // the status word, drains its copies and leaves through the common exit (TMEM is freed).
@@ -40,7 +40,7 @@ namespace qzo {
 namespace {
 
 constexpr int kATmemColsPerStage = kBlockK / 2;   // 64 bf16 along K = 32 TMEM columns of 32 bits
-constexpr int kScaleSlots = 8;        // ring of perturbed-scale rows (one per quantisation group)
+constexpr int kMaxASlots = 4;         // A-ring slots (quantisation groups in flight); each holds its perturbed scales
 constexpr int kNumScaleWarps = 4;
 constexpr int kNumDeqWarps = 8;
 constexpr int kNumEpiWarps = 8;
@@ -277,14 +277,14 @@ struct SmemPlan {
   static constexpr int kPasses = TOK / kPassTok;
   static constexpr int kStagingBufBytes = kPassTok * kTileN * 2;
   static constexpr int kStagingBytes = OUT_MODE == kOutBf16 ? 2 * kStagingBufBytes : 0;
-  static constexpr int kFixedBytes = kStagingBytes + kScaleSlots * kCookedScaleBytes + 1024 + 1024;
+  static constexpr int kFixedBytes = kStagingBytes + kMaxASlots * kCookedScaleBytes + 1024 + 1024;
   // int4 path: the A ring (4 KiB of nibbles + 32 TMEM columns per stage) is as deep as tensor memory
   // allows, the B ring takes the shared memory that is left; bf16 path: both rings alike
   static constexpr int kStagesTmem = (512 - kAccCols) / kATmemColsPerStage;
   // A slot of the int4 path = one quantisation group = two k-blocks: one 8 KiB bulk copy, one wait
   // and one arrival per group for the producer, the de-quantisers and the MMA warp
   static constexpr int kAGroup = DEQUANT ? 2 : 1;                  // k-blocks per A-ring slot
-  static constexpr int kAStages = DEQUANT ? cmin(8, kStagesTmem) / 2 * 2 : 4;
+  static constexpr int kAStages = DEQUANT ? cmin(2 * kMaxASlots, kStagesTmem) / 2 * 2 : 4;
   static constexpr int kASlots = kAStages / kAGroup;
   static constexpr int kBStages = DEQUANT ? cmin(8, (kSmemBudget - kFixedBytes - kAStages * kAStageBytes) / kXTileBytes) : 4;
   static_assert(kBStages >= 2 && kASlots >= 2, "pipelines need at least two stages");
@@ -292,8 +292,8 @@ struct SmemPlan {
   static constexpr int kOffA = kBStages * kXTileBytes;
   static constexpr int kOffStaging = kOffA + kAStages * kAStageBytes;
   static constexpr int kOffCooked = kOffStaging + kStagingBytes;
-  static constexpr int kOffBars = kOffCooked + kScaleSlots * kCookedScaleBytes;
-  static constexpr int kNumBars = 2 * kBStages + 3 * kAStages + 2 * kScaleSlots + 2;
+  static constexpr int kOffBars = kOffCooked + kMaxASlots * kCookedScaleBytes;
+  static constexpr int kNumBars = 2 * kBStages + 3 * kAStages + 2;
   static constexpr int kOffMisc = kOffBars + kNumBars * 8;
   static constexpr int kTotal = kOffMisc + 32;
   static constexpr int kDynamicBytes = kTotal + 1024;      // slack for the 1024-byte alignment
@@ -363,10 +363,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
   auto bar_a_full = [&](int s) { return bar0 + 8u * (2 * kBStages + s); };       // packed nibbles / bf16 weights landed
   auto bar_a_deq = [&](int s) { return bar0 + 8u * (2 * kBStages + kAStages + s); };      // A stage de-quantised
   auto bar_a_empty = [&](int s) { return bar0 + 8u * (2 * kBStages + 2 * kAStages + s); };  // MMAs that read it retired
-  const uint32_t bar_sc0 = bar0 + 8u * (2 * kBStages + 3 * kAStages);
-  auto bar_sc_full = [&](int g) { return bar_sc0 + 8u * g; };
-  auto bar_sc_empty = [&](int g) { return bar_sc0 + 8u * (kScaleSlots + g); };
-  const uint32_t bar_acc_full = bar_sc0 + 8u * (2 * kScaleSlots);                // accumulator complete
+  const uint32_t bar_acc_full = bar0 + 8u * (2 * kBStages + 3 * kAStages);       // accumulator complete
   const uint32_t bar_acc_empty = bar_acc_full + 8u;                              // accumulator drained
   volatile int* const abort_flag = reinterpret_cast<volatile int*>(smem + Plan::kOffMisc);
   uint32_t* const tmem_slot = reinterpret_cast<uint32_t*>(smem + Plan::kOffMisc + 4);
@@ -388,13 +385,10 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
       mbar_init(bar_b_empty(s), 1);
     }
     for (int s = 0; s < kASlots; ++s) {
-      mbar_init(bar_a_full(s), 1);
+      // int4 path: the slot is full when its nibbles have landed AND its perturbed scales are written
+      mbar_init(bar_a_full(s), DEQUANT ? 2 : 1);
       mbar_init(bar_a_deq(s), kNumDeqWarps);
       mbar_init(bar_a_empty(s), 1);
-    }
-    for (int g = 0; g < kScaleSlots; ++g) {
-      mbar_init(bar_sc_full(g), 1);
-      mbar_init(bar_sc_empty(g), kNumDeqWarps);
     }
     mbar_init(bar_acc_full, 1);
     mbar_init(bar_acc_empty, 1);
@@ -513,8 +507,8 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         const int ngroups = (w.nkb + 1) >> 1;
         for (int gi = 0; gi < ngroups; ++gi, ++gig) {
           if ((gig % kNumScaleWarps) != sw) continue;
-          const int slot = gig % kScaleSlots;
-          const uint32_t gph = (uint32_t)(gig / kScaleSlots) & 1u;
+          const int slot = gig % kASlots;                // the A-ring slot of this group
+          const uint32_t gph = (uint32_t)(gig / kASlots) & 1u;
           const int g = (w.kb_begin >> 1) + gi;
           const int r0 = lane * 4;                       // four consecutive output features = one counter block
           float sv[4] = {0.0f, 0.0f, 0.0f, 0.0f};
@@ -540,12 +534,13 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             cooked[2 * l] = h16 | (h16 << 16);
             cooked[2 * l + 1] = l16 | (l16 << 16);
           }
-          if (!__all_sync(0xffffffffu, mbar_wait_relaxed(bar_sc_empty(slot), gph ^ 1u, abort_flag))) { ok = false; break; }
+          // the slot (nibbles, scales, tensor-memory stages) is free once the MMAs of its previous group retired
+          if (!__all_sync(0xffffffffu, mbar_wait_relaxed(bar_a_empty(slot), gph ^ 1u, abort_flag))) { ok = false; break; }
           uint4* dst = reinterpret_cast<uint4*>(smem + Plan::kOffCooked + slot * kCookedScaleBytes + r0 * 8);
           dst[0] = make_uint4(cooked[0], cooked[1], cooked[2], cooked[3]);
           dst[1] = make_uint4(cooked[4], cooked[5], cooked[6], cooked[7]);
           __syncwarp();
-          if (lane == 0) mbar_arrive(bar_sc_full(slot));
+          if (lane == 0) mbar_arrive(bar_a_full(slot));
         }
       }
       if (!ok) *abort_flag = 1;
@@ -577,24 +572,18 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
       // A stage in tensor memory: lane = row (this warp's quadrant), column = k / 2
       const uint32_t a_lane_base = tmem_d + ((uint32_t)((warp & 3) * 32) << 16) + kAccCols + (uint32_t)(h * 16);
       Ring ra;                              // A-ring slot = one quantisation group (two k-blocks)
-      int gig = 0;
       for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x) {
         const Unit w = decode_unit(p, u, TOK);
         for (int it = 0; it < w.nkb; it += 2) {
           const bool two = it + 1 < w.nkb;                    // the last group of an odd K has one k-block
+          // the slot is full: nibbles landed, perturbed scales written; that implies it had been released
+          // by the MMAs that last read it
+          if (!__all_sync(0xffffffffu, mbar_wait(bar_a_full(ra.s), ra.ph, abort_flag))) { ok = false; break; }
           {
-            const int slot = gig % kScaleSlots;
-            const uint32_t gph = (uint32_t)(gig / kScaleSlots) & 1u;
-            ++gig;
-            if (!__all_sync(0xffffffffu, mbar_wait(bar_sc_full(slot), gph, abort_flag))) { ok = false; break; }
-            const uint2 c = *reinterpret_cast<const uint2*>(smem + Plan::kOffCooked + slot * kCookedScaleBytes + r * 8);
+            const uint2 c = *reinterpret_cast<const uint2*>(smem + Plan::kOffCooked + ra.s * kCookedScaleBytes + r * 8);
             *reinterpret_cast<uint32_t*>(&s_hi) = c.x;
             *reinterpret_cast<uint32_t*>(&s_lo) = c.y;
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_sc_empty(slot));
           }
-          // bar_a_full completing implies the slot was released by the MMAs that last read it
-          if (!__all_sync(0xffffffffu, mbar_wait(bar_a_full(ra.s), ra.ph, abort_flag))) { ok = false; break; }
           const uint8_t* src = smem + Plan::kOffA + ra.s * (2 * Plan::kAStageBytes) + (h * kTileN + r) * 16;
           const uint4 pk0 = *reinterpret_cast<const uint4*>(src);
           uint4 pk1 = make_uint4(0, 0, 0, 0);
