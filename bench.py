@@ -112,12 +112,14 @@ def oracle_sample(workload, n_seq=2):
     n_seq = min(n_seq, c["batch"])
     tok, lab = inputs.tokens_and_labels(cfg, n_seq, c["seq"], seed=7)
     lab = np.where(lab.numpy() >= 8, -100, lab.numpy())       # the sample keeps 8 rows of the head only
+    signs = (+1, -1) if n_seq > 1 else (+1,)
     t0 = time.perf_counter()
-    omodel.forward_loss(m, tok.numpy(), lab, 42, +1, c["eps"])
+    for sign in signs:
+        omodel.forward_loss(m, tok.numpy(), lab, 42, sign, c["eps"])
     dt = time.perf_counter() - t0
-    step_s = dt * c["n_layers"] * 2 * (c["batch"] / n_seq)
+    step_s = dt * c["n_layers"] * (2 / len(signs)) * (c["batch"] / n_seq)
     cores = torch.get_num_threads()
-    desc = (f"oracle forward of 1 of {c['n_layers']} decoder blocks, 1 of 2 signs, {n_seq} of {c['batch']} "
+    desc = (f"oracle forward of 1 of {c['n_layers']} decoder blocks, {len(signs)} of 2 signs, {n_seq} of {c['batch']} "
             f"sequences (S={c['seq']}) in {dt:.2f} s; extrapolated linearly to a whole step")
     return 1.0 / step_s, cores, desc
 
