@@ -132,3 +132,33 @@ def test_batch_limits_and_bad_arguments(lib):
     ref = omodel.forward_loss(om, small_tok.cpu().numpy(), small_lab.cpu().numpy(), 3, 0, 1e-3)
     assert abs(loss - ref) <= 1e-3
     gm.close()
+
+
+def test_nonfinite_loss_is_reported_and_leaves_the_scales_untouched(lib):
+    # Training "collapse" shows as a non-finite loss; the step must then report it and change nothing.
+    # The failure is injected on the host (one scale set to NaN), not on the device.
+    cfg, c, om, gm, tok, lab = _setup(lib, "tiny")
+    gm.scales[5] = float("nan")
+    before = gm.scales.clone()
+    with pytest.raises(lib.QzoError) as e:
+        gm.qzo_step(tok.cuda(), lab.cuda(), 42, c["eps"], c["lr"], c["clip"])
+    assert e.value.status == lib.ERR_NONFINITE
+    torch.cuda.synchronize()
+    same = (gm.scales.view(torch.int16) == before.view(torch.int16))
+    assert bool(same.all())
+    assert gm.qzo_device_status() == 0
+    gm.close()
+
+
+def test_empty_and_minimal_calls(lib):
+    # zero-length requests are no-ops; a single token and a single sequence work
+    assert lib.qzo_normals(1, 0, 0).numel() == 0
+    s = torch.full((8,), 0.01, dtype=torch.bfloat16, device="cuda")
+    lib._check(lib._lib.qzo_update_scales_flat(lib._ptr(s), 0, 1, 0, 1e-3, 1.0, 10.0, lib._stream()), "empty update")
+    assert bool((s == 0.01).all())
+    cfg, c, om, gm, tok, lab = _setup(lib, "tiny")
+    t1, l1 = tok[:1, :1].contiguous().cuda(), torch.zeros((1, 1), dtype=torch.int32, device="cuda")
+    loss = float(gm.qzo_forward_loss(t1, l1, 3, +1, 1e-3).cpu()[0])
+    ref = omodel.forward_loss(om, t1.cpu().numpy(), l1.cpu().numpy(), 3, +1, 1e-3)
+    assert abs(loss - ref) <= 1e-3
+    gm.close()
