@@ -395,9 +395,12 @@ __global__ void relu_kernel(__nv_bfloat16* __restrict__ x, int64_t nvec) {
 }
 
 // Row-wise cross entropy on fp32 logits: row_loss[t] = logsumexp(logits[t]) - logits[t][label],
-// 0 and not counted when label == -100.
-__global__ void ce_rows_kernel(const float* __restrict__ logits, const int32_t* __restrict__ labels, int V,
-                               float* __restrict__ row_loss) {
+// 0 and not counted when label == -100.  One pass over the row: every thread keeps a running
+// maximum and a sum of exponentials relative to it (16-byte loads when V is a multiple of 4), the
+// block then merges the (max, sum) pairs in a fixed order.
+__global__ void __launch_bounds__(256)
+ce_rows_kernel(const float* __restrict__ logits, const int32_t* __restrict__ labels, int V,
+               float* __restrict__ row_loss) {
   __shared__ float red[32];
   const int t = blockIdx.x;
   const int label = labels[t];
@@ -406,13 +409,24 @@ __global__ void ce_rows_kernel(const float* __restrict__ logits, const int32_t* 
     return;
   }
   const float* row = logits + (size_t)t * V;
-  float mx = -INFINITY;
-  for (int i = threadIdx.x; i < V; i += blockDim.x) mx = fmaxf(mx, row[i]);
-  mx = block_max(mx, red);
-  float se = 0.0f;
-  for (int i = threadIdx.x; i < V; i += blockDim.x) se += expf(row[i] - mx);
-  se = block_sum(se, red);
-  if (threadIdx.x == 0) row_loss[t] = (mx + logf(se)) - row[label];
+  float mx = -INFINITY, se = 0.0f;
+  auto take = [&](float x) {
+    if (x > mx) { se = se * __expf(mx - x) + 1.0f; mx = x; }
+    else se += __expf(x - mx);
+  };
+  if ((V & 3) == 0) {
+    const float4* row4 = reinterpret_cast<const float4*>(row);
+    for (int i = threadIdx.x; i < (V >> 2); i += blockDim.x) {
+      const float4 v = row4[i];
+      take(v.x); take(v.y); take(v.z); take(v.w);
+    }
+  } else {
+    for (int i = threadIdx.x; i < V; i += blockDim.x) take(row[i]);
+  }
+  const float gmx = block_max(mx, red);
+  const float part = (mx == -INFINITY) ? 0.0f : se * __expf(mx - gmx);
+  const float total = block_sum(part, red);
+  if (threadIdx.x == 0) row_loss[t] = (gmx + logf(total)) - row[label];
 }
 
 // loss = sum(row_loss over kept rows) / count, summed in a fixed order by one block.
