@@ -40,7 +40,7 @@ namespace qzo {
 namespace {
 
 constexpr int kATmemColsPerStage = kBlockK / 2;   // 64 bf16 along K = 32 TMEM columns of 32 bits
-constexpr int kMaxASlots = 4;         // A-ring slots (quantisation groups in flight); each holds its perturbed scales
+constexpr int kMaxASlots = 7;         // A-ring slots (quantisation groups in flight); each holds its perturbed scales
 constexpr int kNumScaleWarps = 4;
 constexpr int kNumDeqWarps = 8;
 constexpr int kNumEpiWarps = 8;
