@@ -16,7 +16,7 @@
 // the activations (q, k, v or gate, up) are served by one launch; the logical scale index of a
 // scale never depends on that grouping.
 //
-// Warp roles (23 warps):
+// Warp roles (24 warps):
 //   warp 0       TMA producer of the B ring: activation tiles (2-D tensor map, 128-byte swizzle)
 //   warp 1       MMA issuer (one elected lane), owns the TMEM allocation
 //   warp 2       producer of the A ring: packed int4 tiles (one 8 KiB bulk copy per quantisation group)
@@ -45,7 +45,8 @@ constexpr int kNumScaleWarps = 4;
 constexpr int kNumDeqWarps = 8;
 constexpr int kNumEpiWarps = 8;
 constexpr int kAProducerWarp = 2;
-constexpr int kFirstScaleWarp = 3;
+constexpr int kWatchWarp = 3;          // waits on the mbarriers on behalf of the MMA issuer
+constexpr int kFirstScaleWarp = 4;
 constexpr int kFirstDeqWarp = kFirstScaleWarp + kNumScaleWarps;
 constexpr int kFirstEpiWarp = kFirstDeqWarp + kNumDeqWarps;
 constexpr int kNumWarps = kFirstEpiWarp + kNumEpiWarps;
@@ -187,6 +188,14 @@ __device__ __forceinline__ bool elect_one() {
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(pred));
   return pred != 0;
+}
+__device__ __forceinline__ int ld_acquire_shared(uint32_t addr) {
+  int v;
+  asm volatile("ld.acquire.cta.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release_shared(uint32_t addr, int v) {
+  asm volatile("st.release.cta.shared.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
 __device__ __forceinline__ void tcgen05_fence_before() {
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -350,6 +359,8 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
   constexpr int kBStages = Plan::kBStages;
   constexpr uint32_t kAccCols = Plan::kAccCols;
   constexpr uint32_t kTmemCols = Plan::kTmemCols;
+  // With 256-token tiles the MMA-issuing thread is the bottleneck: a watch warp does its mbarrier waits.
+  constexpr bool kWatch = TOK == 256;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* const smem = smem_raw + (base - smem_u32(smem_raw));
@@ -372,11 +383,17 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
   // up: it holds the first unit count that must not be started.  Written by that warp only, before it
   // reaches the barrier, so that every warp leaves the loop at the same barrier.
   volatile int* const epi_stop = reinterpret_cast<volatile int*>(smem + Plan::kOffMisc + 12);
+  // Number of k-blocks (of this CTA, all units) whose operands the watch warp has seen ready; -1 when it
+  // gave up.  The MMA issuer reads this word instead of polling mbarriers: a ready mbarrier wait costs
+  // the issuing thread about three times as much as a shared-memory load, and that thread is the
+  // bottleneck of the kernel.
+  const uint32_t ready_addr = base + Plan::kOffMisc + 16;
 
   if (threadIdx.x == 0) {
     *abort_flag = 0;
     *never_set = 0;
     *epi_stop = 0x7fffffff;
+    *reinterpret_cast<volatile int*>(smem + Plan::kOffMisc + 16) = 0;
     for (int s = 0; s < kBStages; ++s) {
       // bf16 path: one barrier tells the MMA warp that both tiles of a stage have landed (rings of
       // equal depth).  int4 path: the A ring is deeper than the B ring, so the de-quantisers signal
@@ -458,16 +475,28 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     // issues the MMAs and the commits.
     constexpr uint32_t idesc = umma_idesc_bf16(kTileN, TOK);
     Ring ra, rb;
-    int useq = 0;
+    int itg = 0, useq = 0;
     for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x, ++useq) {
       const Unit w = decode_unit(p, u, TOK);
-      // the epilogue warps must have drained the previous unit's accumulator
-      if (!mbar_wait(bar_acc_empty, ((uint32_t)useq & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-      tcgen05_fence_after();
-      for (int it = 0; it < w.nkb; ++it) {
+      for (int it = 0; it < w.nkb; ++it, ++itg) {
         const int j = it % kAGroup;                           // position inside the A slot
-        if (DEQUANT && j == 0 && !mbar_wait(bar_a_deq(ra.s), ra.ph, abort_flag)) { ok = false; break; }
-        if (!mbar_wait(bar_b_full(rb.s), rb.ph, abort_flag)) { ok = false; break; }
+        if (!kWatch) {
+          // small token tiles are bound by latency, not by this thread's instruction count: wait here
+          if (it == 0 && !mbar_wait(bar_acc_empty, ((uint32_t)useq & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+          if (DEQUANT && j == 0 && !mbar_wait(bar_a_deq(ra.s), ra.ph, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(bar_b_full(rb.s), rb.ph, abort_flag)) { ok = false; break; }
+        } else {
+          // wait (bounded) until the watch warp has seen this k-block's operands ready and, for the
+          // first k-block of a unit, the accumulator drained
+          int seen = ld_acquire_shared(ready_addr);
+          if (seen >= 0 && seen <= itg) {
+            const long long t0 = clock64();
+            do {
+              seen = ld_acquire_shared(ready_addr);
+            } while (seen >= 0 && seen <= itg && clock64() - t0 < kWaitLimitCycles);
+          }
+          if (seen <= itg) { ok = false; break; }             // the watch warp gave up (-1), or the limit expired
+        }
         tcgen05_fence_after();
         const bool slot_done = j == kAGroup - 1 || it == w.nkb - 1;
         const uint64_t bdesc = umma_desc_k_major_sw128(base + Plan::kOffB + rb.s * Plan::kXTileBytes);
@@ -496,6 +525,36 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
       __syncwarp();
     }
     if (!ok) *abort_flag = 1;
+  } else if (warp == kWatchWarp) {
+    if (kWatch) {
+    // ------------------------------------------------------------------ watch warp
+    // Performs the (bounded) mbarrier waits the MMA issuer depends on, one k-block ahead of it in
+    // time, and publishes the count of ready k-blocks.
+    Ring ra, rb;
+    int useq = 0, itg = 0;
+    for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x, ++useq) {
+      const Unit w = decode_unit(p, u, TOK);
+      for (int it = 0; it < w.nkb; ++it) {
+        const int j = it % kAGroup;
+        bool got = true;
+        // the epilogue warps must have drained the previous unit's accumulator
+        if (it == 0) got = mbar_wait(bar_acc_empty, ((uint32_t)useq & 1u) ^ 1u, abort_flag);
+        if (DEQUANT && j == 0) got = got && mbar_wait(bar_a_deq(ra.s), ra.ph, abort_flag);
+        got = got && mbar_wait(bar_b_full(rb.s), rb.ph, abort_flag);
+        __syncwarp();
+        if (!got) {
+          if (lane == 0) st_release_shared(ready_addr, -1);
+          ok = false;
+          break;
+        }
+        ++itg;
+        if (lane == 0) st_release_shared(ready_addr, itg);
+        if (j == kAGroup - 1 || it == w.nkb - 1) ra.next(kASlots);
+        rb.next(kBStages);
+      }
+    }
+    if (!ok) *abort_flag = 1;
+    }
   } else if (warp < kFirstDeqWarp) {
     // ------------------------------------------------------------------ scale warps
     if (DEQUANT) {
