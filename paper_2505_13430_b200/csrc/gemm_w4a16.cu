@@ -230,6 +230,24 @@ __device__ __forceinline__ void umma_bf16_tmem_a(uint32_t d_tmem, uint32_t a_tme
       ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// The four MMAs of one 64-deep k-block (K = 16 each) with A in tensor memory, in one instruction
+// sequence: A advances by 8 TMEM columns, the B descriptor by 32 bytes (2 in its address field) per
+// step; only the first may overwrite the accumulator.
+__device__ __forceinline__ void umma_bf16_tmem_a_x4(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
+                                                    uint32_t accumulate_first) {
+  asm volatile(
+      "{\n\t.reg .pred p, t;\n\t.reg .b32 a1, a2, a3;\n\t.reg .b64 b1, b2, b3;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "setp.eq.b32 t, 0, 0;\n\t"
+      "add.u32 a1, %1, 8;\n\t add.u32 a2, %1, 16;\n\t add.u32 a3, %1, 24;\n\t"
+      "add.u64 b1, %2, 2;\n\t add.u64 b2, %2, 4;\n\t add.u64 b3, %2, 6;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a1], b1, %3, t;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a2], b2, %3, t;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a3], b3, %3, t;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate_first)
+      : "memory");
+}
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t v[16]) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
@@ -474,6 +492,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     // The whole warp walks the loop (warp-uniform control flow and addresses); one elected lane
     // issues the MMAs and the commits.
     constexpr uint32_t idesc = umma_idesc_bf16(kTileN, TOK);
+    const bool leader = elect_one();
     Ring ra, rb;
     int itg = 0, useq = 0;
     for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x, ++useq) {
@@ -500,13 +519,11 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         tcgen05_fence_after();
         const bool slot_done = j == kAGroup - 1 || it == w.nkb - 1;
         const uint64_t bdesc = umma_desc_k_major_sw128(base + Plan::kOffB + rb.s * Plan::kXTileBytes);
-        if (elect_one()) {
+        if (leader) {
           if (DEQUANT) {
             const uint32_t a_tmem = tmem_d + kAccCols + (uint32_t)((ra.s * kAGroup + j) * kATmemColsPerStage);
-#pragma unroll
-            for (int k = 0; k < kBlockK / 16; ++k)      // 16 bf16 along K = 8 TMEM columns
-              umma_bf16_tmem_a(tmem_d, a_tmem + (uint32_t)(k * 8), bdesc + (uint64_t)(k * 2), idesc,
-                               (it > 0 || k > 0) ? 1u : 0u);
+            static_assert(kBlockK == 64, "four K = 16 steps per k-block");
+            umma_bf16_tmem_a_x4(tmem_d, a_tmem, bdesc, idesc, it > 0 ? 1u : 0u);
           } else {
             const uint64_t adesc = umma_desc_k_major_sw128(base + Plan::kOffA + ra.s * Plan::kAStageBytes);
 #pragma unroll
@@ -521,7 +538,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         if (slot_done) ra.next(kASlots);
         rb.next(kBStages);
       }
-      if (ok && elect_one()) umma_commit(bar_acc_full);
+      if (ok && leader) umma_commit(bar_acc_full);
       __syncwarp();
     }
     if (!ok) *abort_flag = 1;
