@@ -220,16 +220,6 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint6
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-// Same MMA with the A operand read from tensor memory (lane = row, 2 bf16 per 32-bit column).
-__device__ __forceinline__ void umma_bf16_tmem_a(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
-                                                 uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
 // The four MMAs of one 64-deep k-block (K = 16 each) with A in tensor memory, in one instruction
 // sequence: A advances by 8 TMEM columns, the B descriptor by 32 bytes (2 in its address field) per
 // step; only the first may overwrite the accumulator.
@@ -493,6 +483,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     // issues the MMAs and the commits.
     constexpr uint32_t idesc = umma_idesc_bf16(kTileN, TOK);
     const bool leader = elect_one();
+    const uint64_t bdesc0 = umma_desc_k_major_sw128(base + Plan::kOffB);   // stage s: start address + s * tile bytes
     Ring ra, rb;
     int itg = 0, useq = 0;
     for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x, ++useq) {
@@ -518,7 +509,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         }
         tcgen05_fence_after();
         const bool slot_done = j == kAGroup - 1 || it == w.nkb - 1;
-        const uint64_t bdesc = umma_desc_k_major_sw128(base + Plan::kOffB + rb.s * Plan::kXTileBytes);
+        const uint64_t bdesc = bdesc0 + (uint64_t)(rb.s * (Plan::kXTileBytes >> 4));
         if (leader) {
           if (DEQUANT) {
             const uint32_t a_tmem = tmem_d + kAccCols + (uint32_t)((ra.s * kAGroup + j) * kATmemColsPerStage);
@@ -534,7 +525,6 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
           umma_commit(bar_b_empty(rb.s));                 // releases the B stage
           if (slot_done) umma_commit(bar_a_empty(ra.s));  // and, after its last k-block, the A slot
         }
-        __syncwarp();
         if (slot_done) ra.next(kASlots);
         rb.next(kBStages);
       }
