@@ -851,16 +851,30 @@ int launch_tok(int tok, const CUtensorMap& tx, const CUtensorMap& tw, const CUte
 }  // namespace
 
 // Split-K plan: number of K slices for a problem (1 = none).  Slices hold an even number of
-// k-blocks so that they start on a quantisation-group boundary.
+// k-blocks so that they start on a quantisation-group boundary.  The choice minimises a simple
+// cost model measured on B200: a unit costs a pipeline fill plus ~600 cycles per k-block whatever
+// the token tile, the units run in rounds of one per SM, and a split adds the fp32 partial sums'
+// round trip and a second launch.  Depends on the shape only, so results are reproducible.
 int gemm_splits(int M, int K, int N) {
   const int tok = pick_tok_tile(M);
+  if (tok > 128) return 1;                       // 256-token tiles: plenty of units, tensor-bound
   const int tiles = ceil_div(N, kTileN) * ceil_div(M, tok);
   const int groups = ceil_div(K, kGroup);
-  if (tiles >= 120 || groups < 8) return 1;
-  int splits = 296 / tiles;                      // aim at two units per SM
-  if (splits > groups / 4) splits = groups / 4;  // at least four groups per slice
-  if (splits > 16) splits = 16;
-  return splits < 1 ? 1 : splits;
+  const int sms = 148;
+  const double cycles_per_kb = 600.0, fill_cycles = 3500.0, clock_ghz = 1.8;
+  int best = 1;
+  double best_us = 1e30;
+  for (int sp = 1; sp <= 16 && sp <= groups; ++sp) {
+    const int groups_per = ceil_div(groups, sp);
+    if (sp > 1 && groups_per < 4) break;         // at least four groups per slice
+    const int slices = ceil_div(groups, groups_per);
+    if (slices != sp) continue;                  // same partition as a smaller sp
+    const int rounds = ceil_div(tiles * slices, sms);
+    double us = rounds * (groups_per * 2 * cycles_per_kb + fill_cycles) / (clock_ghz * 1e3);
+    if (sp > 1) us += 3.0 + (double)(sp + 1) * M * N * 4.0 / 3.0e6;   // second launch + partial sums at ~3 TB/s
+    if (us < best_us) { best_us = us; best = sp; }
+  }
+  return best;
 }
 
 size_t gemm_workspace_bytes(int M, int K, int N) {

@@ -49,7 +49,7 @@ def test_noalloc_entry_matches_workspace_entry_twice_in_a_row():
 
 def test_noalloc_entry_rejects_problems_beyond_its_scratch():
     from paper_2505_13430_b200 import qzo as lib
-    M, K, N = 128, 4096, 11008                     # partial sums of 16.9 MB exceed the 16 MiB array
+    M, K, N = 128, 8192, 12288                     # split-K partial sums of 18.9 MB exceed the 16 MiB array
     assert lib.qzo_gemm_workspace_bytes(M, K, N) > lib.NOALLOC_SCRATCH_BYTES
     x = torch.zeros((M, K), dtype=torch.bfloat16, device="cuda")
     wq = torch.zeros((lib.qzo_repacked_bytes(K, N),), dtype=torch.uint8, device="cuda")
