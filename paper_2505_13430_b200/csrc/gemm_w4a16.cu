@@ -303,8 +303,12 @@ struct SmemPlan {
   static constexpr int kAGroup = DEQUANT ? 2 : 1;                  // k-blocks per A-ring slot
   static constexpr int kAStages = DEQUANT ? cmin(2 * kMaxASlots, kStagesTmem) / 2 * 2 : 4;
   static constexpr int kASlots = kAStages / kAGroup;
-  static constexpr int kBStages = DEQUANT ? cmin(8, (kSmemBudget - kFixedBytes - kAStages * kAStageBytes) / kXTileBytes) : 4;
-  static_assert(kBStages >= 2 && kASlots >= 2, "pipelines need at least two stages");
+  // Token tiles up to 128: the B ring also works in slots of two k-blocks (one wait, one expect and one
+  // commit per quantisation group); there the per-k-block cost of the single-thread roles is the limit
+  static constexpr int kBGroup = (DEQUANT && TOK <= 128) ? 2 : 1;
+  static constexpr int kBStages = DEQUANT ? cmin(8, (kSmemBudget - kFixedBytes - kAStages * kAStageBytes) / kXTileBytes) / kBGroup * kBGroup : 4;
+  static constexpr int kBSlots = kBStages / kBGroup;
+  static_assert(kBSlots >= 2 && kASlots >= 2, "pipelines need at least two stages");
   static constexpr int kOffB = 0;
   static constexpr int kOffA = kBStages * kXTileBytes;
   static constexpr int kOffStaging = kOffA + kAStages * kAStageBytes;
@@ -365,6 +369,8 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
   constexpr int kASlots = Plan::kASlots;
   constexpr int kAGroup = Plan::kAGroup;
   constexpr int kBStages = Plan::kBStages;
+  constexpr int kBSlots = Plan::kBSlots;
+  constexpr int kBGroup = Plan::kBGroup;
   constexpr uint32_t kAccCols = Plan::kAccCols;
   constexpr uint32_t kTmemCols = Plan::kTmemCols;
   // With 256-token tiles the MMA-issuing thread is the bottleneck: a watch warp does its mbarrier waits.
@@ -402,7 +408,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     *never_set = 0;
     *epi_stop = 0x7fffffff;
     *reinterpret_cast<volatile int*>(smem + Plan::kOffMisc + 16) = 0;
-    for (int s = 0; s < kBStages; ++s) {
+    for (int s = 0; s < kBSlots; ++s) {
       // bf16 path: one barrier tells the MMA warp that both tiles of a stage have landed (rings of
       // equal depth).  int4 path: the A ring is deeper than the B ring, so the de-quantisers signal
       // their own barrier (an arrival on the B barrier could fall into its previous phase)
@@ -432,18 +438,20 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     // warp 0 feeds the B ring (activation tiles), warp 2 the A ring (packed nibbles / bf16 weights)
     if (lane == 0) {
       const bool is_b = warp == 0;
-      const int stages = is_b ? kBStages : kASlots;
+      const int stages = is_b ? kBSlots : kASlots;
       Ring ring;
       int issued = 0;
       for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x) {
         const Unit w = decode_unit(p, u, TOK);
         const LinearDesc& L = p.lin[w.lin];
         if (is_b) {
-          for (int it = 0; it < w.nkb; ++it) {
+          for (int it = 0; it < w.nkb; it += kBGroup) {
+            const int nk = min(kBGroup, w.nkb - it);          // k-blocks of this slot
             if (!mbar_wait(bar_b_empty(ring.s), ring.ph ^ 1u, abort_flag)) { ok = false; break; }
-            mbar_arrive_expect_tx(bar_b_full(ring.s), Plan::kXTileBytes);
-            tma_load_2d(base + Plan::kOffB + ring.s * Plan::kXTileBytes, &tmap_x, bar_b_full(ring.s),
-                        (w.kb_begin + it) * kBlockK, w.tok0);
+            mbar_arrive_expect_tx(bar_b_full(ring.s), (uint32_t)(nk * Plan::kXTileBytes));
+            for (int j = 0; j < nk; ++j)
+              tma_load_2d(base + Plan::kOffB + (ring.s * kBGroup + j) * Plan::kXTileBytes, &tmap_x, bar_b_full(ring.s),
+                          (w.kb_begin + it + j) * kBlockK, w.tok0);
             ring.next(stages);
             ++issued;
           }
@@ -494,7 +502,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
           // small token tiles are bound by latency, not by this thread's instruction count: wait here
           if (it == 0 && !mbar_wait(bar_acc_empty, ((uint32_t)useq & 1u) ^ 1u, abort_flag)) { ok = false; break; }
           if (DEQUANT && j == 0 && !mbar_wait(bar_a_deq(ra.s), ra.ph, abort_flag)) { ok = false; break; }
-          if (!mbar_wait(bar_b_full(rb.s), rb.ph, abort_flag)) { ok = false; break; }
+          if (it % kBGroup == 0 && !mbar_wait(bar_b_full(rb.s), rb.ph, abort_flag)) { ok = false; break; }
         } else {
           // wait (bounded) until the watch warp has seen this k-block's operands ready and, for the
           // first k-block of a unit, the accumulator drained
@@ -509,7 +517,9 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         }
         tcgen05_fence_after();
         const bool slot_done = j == kAGroup - 1 || it == w.nkb - 1;
-        const uint64_t bdesc = bdesc0 + (uint64_t)(rb.s * (Plan::kXTileBytes >> 4));
+        const int jb = it % kBGroup;                          // position inside the B slot
+        const bool bslot_done = jb == kBGroup - 1 || it == w.nkb - 1;
+        const uint64_t bdesc = bdesc0 + (uint64_t)((rb.s * kBGroup + jb) * (Plan::kXTileBytes >> 4));
         if (leader) {
           if (DEQUANT) {
             const uint32_t a_tmem = tmem_d + kAccCols + (uint32_t)((ra.s * kAGroup + j) * kATmemColsPerStage);
@@ -522,11 +532,11 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
               umma_bf16(tmem_d, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
                         (it > 0 || k > 0) ? 1u : 0u);
           }
-          umma_commit(bar_b_empty(rb.s));                 // releases the B stage
+          if (bslot_done) umma_commit(bar_b_empty(rb.s)); // releases the B slot
           if (slot_done) umma_commit(bar_a_empty(ra.s));  // and, after its last k-block, the A slot
         }
         if (slot_done) ra.next(kASlots);
-        rb.next(kBStages);
+        if (bslot_done) rb.next(kBSlots);
       }
       if (ok && leader) umma_commit(bar_acc_full);
       __syncwarp();
@@ -547,7 +557,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         // the epilogue warps must have drained the previous unit's accumulator
         if (it == 0) got = mbar_wait(bar_acc_empty, ((uint32_t)useq & 1u) ^ 1u, abort_flag);
         if (DEQUANT && j == 0) got = got && mbar_wait(bar_a_deq(ra.s), ra.ph, abort_flag);
-        got = got && mbar_wait(bar_b_full(rb.s), rb.ph, abort_flag);
+        if (it % kBGroup == 0) got = got && mbar_wait(bar_b_full(rb.s), rb.ph, abort_flag);
         __syncwarp();
         if (!got) {
           if (lane == 0) st_release_shared(ready_addr, -1);
@@ -557,7 +567,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         ++itg;
         if (lane == 0) st_release_shared(ready_addr, itg);
         if (j == kAGroup - 1 || it == w.nkb - 1) ra.next(kASlots);
-        rb.next(kBStages);
+        if (it % kBGroup == kBGroup - 1 || it == w.nkb - 1) rb.next(kBSlots);
       }
     }
     if (!ok) *abort_flag = 1;
