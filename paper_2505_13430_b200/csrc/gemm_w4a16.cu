@@ -373,8 +373,6 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
   constexpr int kBGroup = Plan::kBGroup;
   constexpr uint32_t kAccCols = Plan::kAccCols;
   constexpr uint32_t kTmemCols = Plan::kTmemCols;
-  // With 256-token tiles the MMA-issuing thread is the bottleneck: a watch warp does its mbarrier waits.
-  constexpr bool kWatch = TOK == 256;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* const smem = smem_raw + (base - smem_u32(smem_raw));
@@ -493,17 +491,12 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     const bool leader = elect_one();
     const uint64_t bdesc0 = umma_desc_k_major_sw128(base + Plan::kOffB);   // stage s: start address + s * tile bytes
     Ring ra, rb;
-    int itg = 0, useq = 0;
-    for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x, ++useq) {
+    int itg = 0;
+    for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x) {
       const Unit w = decode_unit(p, u, TOK);
       for (int it = 0; it < w.nkb; ++it, ++itg) {
         const int j = it % kAGroup;                           // position inside the A slot
-        if (!kWatch) {
-          // small token tiles are bound by latency, not by this thread's instruction count: wait here
-          if (it == 0 && !mbar_wait(bar_acc_empty, ((uint32_t)useq & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-          if (DEQUANT && j == 0 && !mbar_wait(bar_a_deq(ra.s), ra.ph, abort_flag)) { ok = false; break; }
-          if (it % kBGroup == 0 && !mbar_wait(bar_b_full(rb.s), rb.ph, abort_flag)) { ok = false; break; }
-        } else {
+        {
           // wait (bounded) until the watch warp has seen this k-block's operands ready and, for the
           // first k-block of a unit, the accumulator drained
           int seen = ld_acquire_shared(ready_addr);
@@ -543,7 +536,6 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     }
     if (!ok) *abort_flag = 1;
   } else if (warp == kWatchWarp) {
-    if (kWatch) {
     // ------------------------------------------------------------------ watch warp
     // Performs the (bounded) mbarrier waits the MMA issuer depends on, one k-block ahead of it in
     // time, and publishes the count of ready k-blocks.
@@ -571,7 +563,6 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
       }
     }
     if (!ok) *abort_flag = 1;
-    }
   } else if (warp < kFirstDeqWarp) {
     // ------------------------------------------------------------------ scale warps
     if (DEQUANT) {
