@@ -60,7 +60,7 @@ def test_sweep_shapes_match_oracle_on_sampled_outputs(lib, M, K, N):
         assert bool(torch.isfinite(y.float()).all())
 
 
-@pytest.mark.parametrize("workload", ["llama7b", "opt6.7b"])
+@pytest.mark.parametrize("workload", ["llama7b", "llama13b", "opt6.7b"])
 def test_full_width_block_matches_oracle_on_sampled_sequences(lib, workload):
     c = inputs.CONFIGS[workload]
     cfg = inputs.model_cfg(workload, n_layers=1)
