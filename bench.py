@@ -250,7 +250,10 @@ def main():
     shapes = inputs.linear_shapes(cfg)
     T = B * S
     launches_per_layer = 4 if cfg["arch"] == "llama" else 4          # qkv, o, (gate+up | fc1), (down | fc2)
-    mean_bytes = sum(gemm_bytes(T, K, N) for _, K, N in shapes) / launches_per_layer
+    # a step runs its two passes as one forward over both copies of the batch when the token count
+    # allows it: then a launch covers 2 T rows (seen from the number of profiled launches)
+    passes_per_launch = 2 if n_l <= launches_per_layer * cfg["n_layers"] * args.steps else 1
+    mean_bytes = sum(gemm_bytes(passes_per_launch * T, K, N) for _, K, N in shapes) / launches_per_layer
     traffic = NCU_TRAFFIC_RATIO * mean_bytes if NCU_TRAFFIC_RATIO else None
     peaks = measured_peaks()
     value = replicas.whole_job_rate(args.steps, world, ms)

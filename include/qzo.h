@@ -165,7 +165,8 @@ int qzo_scale_layout(const qzo_model_desc* desc, int layer, int linear,
                      int64_t* index_base, int* G, int* N);
 
 /* Bytes of workspace qzo_init_model needs for batches up to max_tokens = B*S tokens
- * (kernel-layout weights + activations + fp32 logits + split-K partials). */
+ * (kernel-layout weights + activations + fp32 logits + split-K partials).  The activation
+ * buffers hold 2 * max_tokens rows, because qzo_step runs both passes as one forward. */
 int qzo_workspace_bytes(const qzo_model_desc* desc, int max_tokens, size_t* bytes);
 
 /* Binds a model to caller-owned tensors (Algorithm 1 "Require": scales Delta, integer
@@ -194,7 +195,11 @@ int qzo_forward_loss(qzo_model* m, const int32_t* d_tokens, const int32_t* d_lab
 int qzo_update_scales(qzo_model* m, uint64_t seed, float lr, float g, float clip);
 
 /* Whole step of Algorithm 1 on device-resident tokens: two forwards (sign +1, -1), d, d' and
- * the update, with d formed on the device.  h_out (may be NULL): {l+, l-, d, d'}; when
+ * the update, with d formed on the device.  When B*S is a multiple of the GEMM's token tile the
+ * two forwards run as ONE pass over two copies of the batch (rows of the second copy take
+ * -eps z); every kernel works row by row or sequence by sequence, so the losses are the ones two
+ * separate passes give, bit for bit, when both use the same token tile (B*S >= 256).
+ * h_out (may be NULL): {l+, l-, d, d'}; when
  * non-NULL the call synchronises the stream.  If either loss is not finite the scales are
  * left untouched and (when h_out is given) QZO_ERR_NONFINITE is returned. */
 int qzo_step(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S,

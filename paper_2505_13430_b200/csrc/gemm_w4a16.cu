@@ -78,6 +78,7 @@ struct GemmParams {
   int splits, m_tiles, total_units;
   unsigned long long seed;
   float sign_eps;                 // sign * eps (0 when unperturbed)
+  int pair_rows;                  // > 0: token rows from this one on take -sign_eps (both passes of a step in one launch)
   int* status;
 };
 
@@ -588,8 +589,10 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
               float z[4];
               const uint64_t i0 = L.idx_base + (uint64_t)g * (uint64_t)L.N + (uint64_t)(w.n0 + r0);
               normals_of_block(p.seed, i0 >> 2, z);
+              // token tiles never straddle pair_rows (checked on the host)
+              const float se = (p.pair_rows > 0 && w.tok0 >= p.pair_rows) ? -p.sign_eps : p.sign_eps;
 #pragma unroll
-              for (int l = 0; l < 4; ++l) sv[l] = fmaf(p.sign_eps, z[l], sv[l]);
+              for (int l = 0; l < 4; ++l) sv[l] = fmaf(se, z[l], sv[l]);
             }
           }
           uint32_t cooked[8];
@@ -878,6 +881,12 @@ int gemm_splits(int M, int K, int N) {
   return best;
 }
 
+// Whether a launch over M token rows may switch the perturbation sign at row `pair_rows`: the
+// boundary must fall between two token tiles.
+bool paired_rows_ok(int M, int pair_rows) {
+  return pair_rows > 0 && pair_rows < M && pair_rows % pick_tok_tile(M) == 0;
+}
+
 size_t gemm_workspace_bytes(int M, int K, int N) {
   const int splits = gemm_splits(M, K, N);
   if (splits <= 1) return 0;
@@ -886,10 +895,13 @@ size_t gemm_workspace_bytes(int M, int K, int N) {
 
 // Y_j = X W'_j (+ bias_j) for up to three linears that share X, with W'_j de-quantised
 // from int4 and perturbed scales.
+// pair_rows > 0: rows [0, pair_rows) are perturbed with sign * eps, rows [pair_rows, M) with -sign * eps;
+// pair_rows must be a multiple of the token tile of M (see paired_rows_ok).
 int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const GemmLinear* lins, int n_lin,
-                                uint64_t seed, int sign, float eps, void* d_ws, size_t ws_bytes, int* d_status,
-                                cudaStream_t st) {
+                                uint64_t seed, int sign, float eps, int pair_rows, void* d_ws, size_t ws_bytes,
+                                int* d_status, cudaStream_t st) {
   if (M <= 0 || K <= 0 || (K % 8) != 0 || n_lin < 1 || n_lin > kMaxGroupedLinears) return QZO_ERR_BAD_ARG;
+  if (pair_rows != 0 && !paired_rows_ok(M, pair_rows)) return QZO_ERR_BAD_ARG;
   for (int j = 0; j < n_lin; ++j)
     if (lins[j].N <= 0 || (lins[j].N % 8) != 0 || (lins[j].idx_base % 4) != 0 || (lins[j].ldo % 8) != 0)
       return QZO_ERR_BAD_ARG;
@@ -900,7 +912,8 @@ int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const Ge
     for (int j = 0; j < n_lin; ++j) any_split = any_split || gemm_splits(M, K, lins[j].N) > 1;
     if (any_split) {
       for (int j = 0; j < n_lin; ++j)
-        QZO_TRY(launch_perturbed_gemm_group(d_x, M, K, lins + j, 1, seed, sign, eps, d_ws, ws_bytes, d_status, st));
+        QZO_TRY(launch_perturbed_gemm_group(d_x, M, K, lins + j, 1, seed, sign, eps, pair_rows, d_ws, ws_bytes, d_status,
+                                            st));
       return QZO_OK;
     }
   }
@@ -913,6 +926,7 @@ int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const Ge
   p.m_tiles = ceil_div(M, tok);
   p.seed = seed;
   p.sign_eps = (float)sign * eps;
+  p.pair_rows = pair_rows;
   p.status = d_status;
   const int splits = (n_lin == 1) ? gemm_splits(M, K, lins[0].N) : 1;
   for (int j = 0; j < n_lin; ++j) {
@@ -1030,7 +1044,7 @@ extern "C" int qzo_perturbed_gemm_noalloc(const void* d_x_bf16, const void* d_wq
   QZO_TRY(noalloc_scratch_address(&scratch));
   const qzo::GemmLinear g{d_wq, (const __nv_bfloat16*)d_scales_bf16, d_bias, (__nv_bfloat16*)d_y_bf16, N, N,
                           scale_index_base};
-  return qzo::launch_perturbed_gemm_group((const __nv_bfloat16*)d_x_bf16, M, K, &g, 1, seed, sign, eps, scratch,
+  return qzo::launch_perturbed_gemm_group((const __nv_bfloat16*)d_x_bf16, M, K, &g, 1, seed, sign, eps, 0, scratch,
                                           (size_t)QZO_NOALLOC_SCRATCH_BYTES, d_status, (cudaStream_t)stream);
 }
 

@@ -133,7 +133,10 @@ struct WsPlan {
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-int plan_workspace(const qzo_model_desc& d, int T, WsPlan* p) {
+// Activation buffers hold twice the caller's token limit: a step runs its two passes (perturbation
+// signs +1 and -1) as one forward over both copies of the batch.
+int plan_workspace(const qzo_model_desc& d, int max_tokens, WsPlan* p) {
+  const int T = 2 * max_tokens;
   LinearShape ls[7];
   const int nl = linear_shapes(d, ls);
   size_t off = 0;
@@ -157,7 +160,8 @@ int plan_workspace(const qzo_model_desc& d, int T, WsPlan* p) {
   p->off_tok = take((size_t)T * 4);
   p->off_lab = take((size_t)T * 4);
   size_t gb = 0;
-  for (int i = 0; i < nl; ++i) gb = std::max(gb, gemm_workspace_bytes(T, ls[i].K, ls[i].N));
+  for (int i = 0; i < nl; ++i)
+    gb = std::max(gb, std::max(gemm_workspace_bytes(T, ls[i].K, ls[i].N), gemm_workspace_bytes(max_tokens, ls[i].K, ls[i].N)));
   p->gemm_bytes = gb;
   p->off_gemm = take(gb);
   p->total = off;
@@ -175,7 +179,7 @@ static int add_norm(qzo_model* m, __nv_bfloat16* x, const __nv_bfloat16* delta, 
 
 // Up to three block linears that read the same input, in one launch.
 static int linears(qzo_model* m, const Linear* const* Ls, __nv_bfloat16* const* outs, int n, int ldo,
-                   const __nv_bfloat16* in, int T, uint64_t seed, int sign, float eps) {
+                   const __nv_bfloat16* in, int T, uint64_t seed, int sign, float eps, int pair_rows) {
   GemmLinear g[kMaxGroupedLinears];
   double flops = 0.0;
   for (int j = 0; j < n; ++j) {
@@ -185,8 +189,8 @@ static int linears(qzo_model* m, const Linear* const* Ls, __nv_bfloat16* const* 
   }
   const bool timed = m->profiling && m->events_used + 2 <= m->events.size();
   if (timed) QZO_CUDA_TRY(cudaEventRecord(m->events[m->events_used], m->stream));
-  QZO_TRY(launch_perturbed_gemm_group(in, T, Ls[0]->K, g, n, seed, sign, eps, m->gemm_ws, m->gemm_ws_bytes, m->status,
-                                      m->stream));
+  QZO_TRY(launch_perturbed_gemm_group(in, T, Ls[0]->K, g, n, seed, sign, eps, pair_rows, m->gemm_ws, m->gemm_ws_bytes,
+                                      m->status, m->stream));
   if (timed) {
     QZO_CUDA_TRY(cudaEventRecord(m->events[m->events_used + 1], m->stream));
     m->events_used += 2;
@@ -195,16 +199,23 @@ static int linears(qzo_model* m, const Linear* const* Ls, __nv_bfloat16* const* 
   return QZO_OK;
 }
 static int linear(qzo_model* m, const Linear& L, const __nv_bfloat16* in, __nv_bfloat16* out, int ldo, int T,
-                  uint64_t seed, int sign, float eps) {
+                  uint64_t seed, int sign, float eps, int pair_rows) {
   const Linear* Ls[1] = {&L};
   __nv_bfloat16* outs[1] = {out};
-  return linears(m, Ls, outs, 1, ldo, in, T, seed, sign, eps);
+  return linears(m, Ls, outs, 1, ldo, in, T, seed, sign, eps, pair_rows);
 }
 
+// One forward pass and its loss.  paired: the batch is given twice (2 B sequences); the first copy
+// is run with sign * eps, the second with -sign * eps, and d_loss[0], d_loss[1] receive the two mean
+// losses.  Every kernel works row by row or sequence by sequence, so each half computes exactly what
+// a pass of its own would.
 int forward_loss(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S, uint64_t seed, int sign,
-                 float eps, float* d_loss) {
+                 float eps, float* d_loss, bool paired) {
   const qzo_model_desc& d = m->desc;
-  const int T = B * S, dm = d.d_model, H = d.n_heads, dh = dm / H, F = d.d_ffn;
+  const int dm = d.d_model, H = d.n_heads, dh = dm / H, F = d.d_ffn;
+  const int pair_rows = paired ? B * S : 0;
+  if (paired) B *= 2;
+  const int T = B * S;
   cudaStream_t st = m->stream;
   const bool llama = d.arch == QZO_ARCH_LLAMA;
   QZO_TRY(launch_embedding(d_tokens, m->embed, llama ? nullptr : m->pos_embed, T, S, dm, d.vocab, m->x, st));
@@ -219,22 +230,22 @@ int forward_loss(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels,
     {
       const Linear* qkv_l[3] = {&L.lin[0], &L.lin[1], &L.lin[2]};
       __nv_bfloat16* qkv_o[3] = {m->qkv, m->qkv + dm, m->qkv + 2 * dm};
-      QZO_TRY(linears(m, qkv_l, qkv_o, 3, 3 * dm, m->xn, T, seed, sign, eps));
+      QZO_TRY(linears(m, qkv_l, qkv_o, 3, 3 * dm, m->xn, T, seed, sign, eps, pair_rows));
     }
     if (llama) QZO_TRY(launch_rope(m->qkv, m->qkv + dm, 3 * dm, 3 * dm, m->rope_cs, T, S, H, dh, st));
     QZO_TRY(launch_attention(m->qkv, m->qkv + dm, m->qkv + 2 * dm, 3 * dm, 3 * dm, 3 * dm, m->att, dm, B, S, H, dh, st));
-    QZO_TRY(linear(m, L.lin[3], m->att, m->xn, dm, T, seed, sign, eps));
+    QZO_TRY(linear(m, L.lin[3], m->att, m->xn, dm, T, seed, sign, eps, pair_rows));
     QZO_TRY(add_norm(m, m->x, m->xn, L.norm2_w, L.norm2_b, T, m->xn));
     if (llama) {
       const Linear* gu_l[2] = {&L.lin[4], &L.lin[5]};
       __nv_bfloat16* gu_o[2] = {m->mlp_a, m->mlp_b};
-      QZO_TRY(linears(m, gu_l, gu_o, 2, F, m->xn, T, seed, sign, eps));
+      QZO_TRY(linears(m, gu_l, gu_o, 2, F, m->xn, T, seed, sign, eps, pair_rows));
       QZO_TRY(launch_silu_mul(m->mlp_a, m->mlp_b, m->mlp_a, (int64_t)T * F, st));
-      QZO_TRY(linear(m, L.lin[6], m->mlp_a, m->xn, dm, T, seed, sign, eps));
+      QZO_TRY(linear(m, L.lin[6], m->mlp_a, m->xn, dm, T, seed, sign, eps, pair_rows));
     } else {
-      QZO_TRY(linear(m, L.lin[4], m->xn, m->mlp_a, F, T, seed, sign, eps));
+      QZO_TRY(linear(m, L.lin[4], m->xn, m->mlp_a, F, T, seed, sign, eps, pair_rows));
       QZO_TRY(launch_relu(m->mlp_a, (int64_t)T * F, st));
-      QZO_TRY(linear(m, L.lin[5], m->mlp_a, m->xn, dm, T, seed, sign, eps));
+      QZO_TRY(linear(m, L.lin[5], m->mlp_a, m->xn, dm, T, seed, sign, eps, pair_rows));
     }
     pending = m->xn;
   }
@@ -242,7 +253,14 @@ int forward_loss(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels,
   if (d.n_layers - 1 == m->capture_layer)
     QZO_CUDA_TRY(cudaMemcpyAsync(m->capture, m->x, (size_t)T * dm * 2, cudaMemcpyDeviceToDevice, st));
   QZO_TRY(launch_bf16_gemm_f32out(m->xn, m->lm_head, m->logits, T, dm, d.vocab, m->status, st));
-  QZO_TRY(launch_cross_entropy(m->logits, d_labels, T, d.vocab, m->row_loss, d_loss, st));
+  if (paired) {
+    const int Th = pair_rows;
+    QZO_TRY(launch_cross_entropy(m->logits, d_labels, Th, d.vocab, m->row_loss, d_loss, st));
+    QZO_TRY(launch_cross_entropy(m->logits + (size_t)Th * d.vocab, d_labels + Th, Th, d.vocab, m->row_loss + Th,
+                                 d_loss + 1, st));
+  } else {
+    QZO_TRY(launch_cross_entropy(m->logits, d_labels, T, d.vocab, m->row_loss, d_loss, st));
+  }
   m->last_T = T;
   return QZO_OK;
 }
@@ -260,8 +278,21 @@ int update_all_scales(qzo_model* m, uint64_t seed, float coef_host, const float*
 
 int step_device(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S, uint64_t seed, float eps,
                 float lr, float clip, float* h_out) {
-  QZO_TRY(forward_loss(m, d_tokens, d_labels, B, S, seed, +1, eps, m->loss2));
-  QZO_TRY(forward_loss(m, d_tokens, d_labels, B, S, seed, -1, eps, m->loss2 + 1));
+  const int T = B * S;
+  if (paired_rows_ok(2 * T, T)) {
+    // both passes as one forward over two copies of the batch (the workspace holds 2 * max_tokens rows)
+    const size_t bytes = (size_t)T * sizeof(int32_t);
+    if (d_tokens != m->tok_dev)
+      QZO_CUDA_TRY(cudaMemcpyAsync(m->tok_dev, d_tokens, bytes, cudaMemcpyDeviceToDevice, m->stream));
+    if (d_labels != m->lab_dev)
+      QZO_CUDA_TRY(cudaMemcpyAsync(m->lab_dev, d_labels, bytes, cudaMemcpyDeviceToDevice, m->stream));
+    QZO_CUDA_TRY(cudaMemcpyAsync(m->tok_dev + T, m->tok_dev, bytes, cudaMemcpyDeviceToDevice, m->stream));
+    QZO_CUDA_TRY(cudaMemcpyAsync(m->lab_dev + T, m->lab_dev, bytes, cudaMemcpyDeviceToDevice, m->stream));
+    QZO_TRY(forward_loss(m, m->tok_dev, m->lab_dev, B, S, seed, +1, eps, m->loss2, true));
+  } else {
+    QZO_TRY(forward_loss(m, d_tokens, d_labels, B, S, seed, +1, eps, m->loss2, false));
+    QZO_TRY(forward_loss(m, d_tokens, d_labels, B, S, seed, -1, eps, m->loss2 + 1, false));
+  }
   QZO_TRY(launch_ddc(m->loss2, m->loss2 + 1, eps, lr, clip, m->out5, m->stream));
   QZO_TRY(update_all_scales(m, seed, 0.0f, m->out5 + 4));
   if (h_out) {
@@ -361,7 +392,7 @@ int qzo_perturbed_gemm(const void* d_x_bf16, const void* d_wq, const void* d_sca
   if (N <= 0 || (N % 8)) return QZO_ERR_BAD_ARG;
   const GemmLinear g{d_wq, (const __nv_bfloat16*)d_scales_bf16, d_bias, (__nv_bfloat16*)d_y_bf16, N, N,
                      scale_index_base};
-  return launch_perturbed_gemm_group((const __nv_bfloat16*)d_x_bf16, M, K, &g, 1, seed, sign, eps, d_workspace,
+  return launch_perturbed_gemm_group((const __nv_bfloat16*)d_x_bf16, M, K, &g, 1, seed, sign, eps, 0, d_workspace,
                                      workspace_bytes, d_status, (cudaStream_t)stream);
 }
 
@@ -544,7 +575,7 @@ int qzo_forward_loss(qzo_model* m, const int32_t* d_tokens, const int32_t* d_lab
                      int sign, float eps, float* d_loss) {
   QZO_TRY(check_batch(m, d_tokens, d_labels, B, S));
   if (!d_loss || sign < -1 || sign > 1 || !(eps > 0.0f)) return QZO_ERR_BAD_ARG;
-  return forward_loss(m, d_tokens, d_labels, B, S, seed, sign, eps, d_loss);
+  return forward_loss(m, d_tokens, d_labels, B, S, seed, sign, eps, d_loss, false);
 }
 
 int qzo_update_scales(qzo_model* m, uint64_t seed, float lr, float g, float clip) {
