@@ -3,12 +3,16 @@
     python -m paper_2505_13430_b200.gemm_sweep [--shapes KxN,...] [--tokens M,...] [--iters I] [--json]
 
 For every shape it times qzo_perturbed_gemm with CUDA events around replays of a CUDA graph that
-holds `iters` launches, rotating through enough distinct weight / scale / activation sets that
-every launch streams its operands from HBM (the rotation exceeds the L2 capacity), and prints the achieved fraction of the roofline
+holds up to `iters` launches (a pass of about 4 ms, at least one launch per set), rotating through
+enough distinct weight / scale / activation sets that every launch streams its operands from HBM
+(the rotation exceeds the L2 capacity).  Every shape is timed alone after an idle second, nine
+passes one by one; the median pass gives the achieved fraction of the roofline
 max(bytes / HBM bandwidth, flops / dense bf16 peak) with
-bytes = K N / 2 + 2 ceil(K/128) N + 2 M K + 2 M N and flops = 2 M K N.
+bytes = K N / 2 + 2 ceil(K/128) N + 2 M K + 2 M N and flops = 2 M K N, against the burst peaks
+(measured the same way: short runs of one kernel); the best pass is printed beside it.
 """
 import argparse
+import time
 import json
 import os
 
@@ -32,7 +36,7 @@ def gemm_bytes(M, K, N):
     return K * N // 2 + 2 * ((K + 127) // 128) * N + 2 * M * K + 2 * M * N
 
 
-def run_shape(M, K, N, iters, sign=1, reps=5):
+def run_shape(M, K, N, iters, sign=1, reps=9, settle=1.0, pass_ms=4.0):
     per_set = gemm_bytes(M, K, N)
     n_sets = max(2, min(64, (2 * L2_BYTES) // per_set + 1))
     sets = []
@@ -56,24 +60,41 @@ def run_shape(M, K, N, iters, sign=1, reps=5):
     for i in range(max(3, n_sets)):
         call(i)
     torch.cuda.synchronize()
+    # One launch, timed with events, sizes the timed pass: a pass rotates through every set at least
+    # once and lasts about `pass_ms`, short enough to be a burst like the one the peak was taken in.
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    call(0)
+    ev1.record()
+    torch.cuda.synchronize()
+    est_us = max(ev0.elapsed_time(ev1) * 1e3, 1.0)
+    iters = max(n_sets, min(iters, int(pass_ms * 1e3 / est_us) + 1))
     # The launches of one timed pass are recorded into a CUDA graph and replayed, so that the
     # figure is device time: at small M a launch from Python costs more than the kernel runs.
     side = torch.cuda.Stream()
     graph = torch.cuda.CUDAGraph()
+    times = []
     with torch.cuda.stream(side):
         with torch.cuda.graph(graph, stream=side):
             for i in range(iters):
                 call(i)
         graph.replay()
         side.synchronize()
-        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        ev0.record(side)
-        for _ in range(reps):
-            graph.replay()
-        ev1.record(side)
+        # Every shape is timed alone, against the burst peaks: an idle moment lets the SM clock recover
+        # from the power-capped run of the shape before it; one untimed replay then warms up again.
+        time.sleep(settle)
+        graph.replay()
         side.synchronize()
+        for _ in range(reps):
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ev0.record(side)
+            graph.replay()
+            ev1.record(side)
+            side.synchronize()
+            times.append(ev0.elapsed_time(ev1) * 1e3 / iters)
     assert int(status.item()) == 0
-    return ev0.elapsed_time(ev1) * 1e3 / (iters * reps), n_sets      # microseconds per launch
+    times.sort()
+    return times[len(times) // 2], times[0], n_sets      # microseconds per launch: median and best pass
 
 
 def main():
@@ -81,6 +102,7 @@ def main():
     ap.add_argument("--shapes", default=",".join(f"{k}x{n}" for k, n in inputs.GEMM_SWEEP_KN))
     ap.add_argument("--tokens", default=",".join(str(m) for m in inputs.GEMM_SWEEP_M))
     ap.add_argument("--iters", type=int, default=50)
+    ap.add_argument("--settle", type=float, default=1.0, help="idle seconds before each shape is timed")
     ap.add_argument("--json", action="store_true")
     args = ap.parse_args()
     bw, tf, src = peaks()
@@ -88,17 +110,18 @@ def main():
     for shape in args.shapes.split(","):
         K, N = (int(v) for v in shape.split("x"))
         for M in (int(v) for v in args.tokens.split(",")):
-            us, n_sets = run_shape(M, K, N, args.iters)
+            us, best_us, n_sets = run_shape(M, K, N, args.iters, settle=args.settle)
             t_hbm = gemm_bytes(M, K, N) / (bw * 1e9) * 1e6
             t_mma = 2.0 * M * K * N / (tf * 1e12) * 1e6
             roof = max(t_hbm, t_mma)
             rows.append({"K": K, "N": N, "M": M, "us": us, "roofline_us": roof, "bound": "hbm" if t_hbm > t_mma else "tensor",
                          "frac": roof / us, "tflops": 2.0 * M * K * N / us / 1e6, "gbs": gemm_bytes(M, K, N) / us / 1e3,
-                         "rotation_sets": n_sets})
+                         "best_pass_us": best_us, "rotation_sets": n_sets})
             r = rows[-1]
             if not args.json:
                 print(f"K={K:6d} N={N:6d} M={M:5d}  {us:9.2f} us  roofline {roof:8.2f} us ({r['bound']:6s})  "
-                      f"frac {r['frac']:.3f}  {r['tflops']:8.1f} TFLOP/s  {r['gbs']:8.1f} GB/s  sets={n_sets}", flush=True)
+                      f"frac {r['frac']:.3f}  {r['tflops']:8.1f} TFLOP/s  {r['gbs']:8.1f} GB/s  best pass {best_us:8.2f} us  sets={n_sets}",
+                      flush=True)
     if args.json:
         print(json.dumps({"peaks": {"hbm_gbs": bw, "bf16_tflops": tf, "source": src}, "rows": rows}))
 
