@@ -16,15 +16,17 @@
 // the activations (q, k, v or gate, up) are served by one launch; the logical scale index of a
 // scale never depends on that grouping.
 //
-// Warp roles (24 warps):
+// Warp roles (25 warps):
 //   warp 0       TMA producer of the B ring: activation tiles (2-D tensor map, 128-byte swizzle)
 //   warp 1       MMA issuer (one elected lane), owns the TMEM allocation
 //   warp 2       producer of the A ring: packed int4 tiles (one 8 KiB bulk copy per quantisation group)
-//   warps 3-6    scale warps: Philox4x32-10 + Box-Muller, s' = s + sign eps z in fp32, split
+//   warp 3       watch warp: does the mbarrier waits the issuer depends on and publishes a count
+//   warps 4-7    scale warps: Philox4x32-10 + Box-Muller, s' = s + sign eps z in fp32, split
 //                into bf16 hi + lo parts, written next to the nibbles of the group's A slot
-//   warps 7-14   de-quantisers: nibbles -> bf16 (u - 8) * s' written to the A stages in TMEM
-//   warps 15-22  epilogue: TMEM -> registers (+ bias) -> bf16 rows in shared memory -> TMA stores;
-//                runs while the other warps already work on the next unit
+//   warps 8-15   de-quantisers: nibbles -> bf16 (u - 8) * s' written to the A stages in TMEM
+//   warps 16-23  epilogue: TMEM -> registers (+ bias) -> bf16 rows in shared memory, 32 tokens per pass
+//   warp 24      store warp: issues the TMA store of every staged pass (three staging buffers), so
+//                that the warps draining the single accumulator never wait for a store to be issued
 // Every wait on an mbarrier is bounded; when a wait expires the CTA records an error in
 // the status word, drains its copies and leaves through the common exit (TMEM is freed).
 #include "qzo_common.cuh"
@@ -49,7 +51,8 @@ constexpr int kWatchWarp = 3;          // waits on the mbarriers on behalf of th
 constexpr int kFirstScaleWarp = 4;
 constexpr int kFirstDeqWarp = kFirstScaleWarp + kNumScaleWarps;
 constexpr int kFirstEpiWarp = kFirstDeqWarp + kNumDeqWarps;
-constexpr int kNumWarps = kFirstEpiWarp + kNumEpiWarps;
+constexpr int kStoreWarp = kFirstEpiWarp + kNumEpiWarps;   // issues the TMA stores of the finished tiles
+constexpr int kNumWarps = kStoreWarp + 1;
 constexpr int kThreads = kNumWarps * 32;
 constexpr long long kWaitLimitCycles = 4000000000LL;   // ~2 s at boost clock
 constexpr int kSmemBudget = 227 * 1024;
@@ -170,7 +173,9 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t sr
       : "memory");
 }
 __device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_group_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// Waits until at most N of this thread's most recent bulk-copy groups still read their source.
+template <int N>
+__device__ __forceinline__ void bulk_wait_group_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
 __device__ __forceinline__ void bulk_wait_group0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
@@ -283,8 +288,8 @@ constexpr int cmin(int a, int b) { return a < b ? a : b; }
 
 // Two rings feed the MMA.  The A ring (packed nibbles in shared memory -> de-quantised bf16 in
 // tensor memory) is deep and cheap, so the de-quantisers run well ahead of the tensor pipe; the
-// B ring holds the activation tiles.  A finished bf16 tile leaves in passes of up to 64 tokens
-// through two staging buffers, each pass as one TMA store.
+// B ring holds the activation tiles.  A finished bf16 tile leaves in passes of up to 32 tokens
+// through three staging buffers, each pass as one TMA store.
 template <int TOK, bool DEQUANT, int OUT_MODE>
 struct SmemPlan {
   static constexpr int kAccCols = TOK < 32 ? 32 : TOK;
@@ -294,7 +299,9 @@ struct SmemPlan {
   static constexpr int kPassTok = TOK < 32 ? TOK : 32;
   static constexpr int kPasses = TOK / kPassTok;
   static constexpr int kStagingBufBytes = kPassTok * kTileN * 2;
-  static constexpr int kStagingBytes = OUT_MODE == kOutBf16 ? 2 * kStagingBufBytes : 0;
+  // three staging buffers: a pass waits for the TMA store issued two passes earlier, not for the last one
+  static constexpr int kStagingBufs = 3;
+  static constexpr int kStagingBytes = OUT_MODE == kOutBf16 ? kStagingBufs * kStagingBufBytes : 0;
   static constexpr int kFixedBytes = kStagingBytes + kMaxASlots * kCookedScaleBytes + 1024 + 1024;
   // int4 path: the A ring (4 KiB of nibbles + 32 TMEM columns per stage) is as deep as tensor memory
   // allows, the B ring takes the shared memory that is left; bf16 path: both rings alike
@@ -431,6 +438,8 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
   const uint32_t tmem_d = *tmem_slot;
 
   bool ok = true;
+  // threads at the epilogue's hardware barrier: for bf16 tiles the store warp takes part
+  constexpr int kEpiBarThreads = (kNumEpiWarps + (OUT_MODE == kOutBf16 ? 1 : 0)) * 32;
 
   if (warp == 0 || warp == kAProducerWarp) {
     // ------------------------------------------------------------------ TMA producers
@@ -675,10 +684,41 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
       }
       if (!ok) *abort_flag = 1;
     }
+  } else if (warp == kStoreWarp) {
+    // ------------------------------------------------------------------ store warp (bf16 tiles)
+    // Walks the units and passes like the epilogue warps and meets them at their hardware barrier:
+    // once a pass is staged, one lane issues its TMA store, so that issuing the store (some hundred
+    // cycles) is off the path of the warps that drain the accumulator.  Before it comes back to the
+    // barrier it waits until the store issued two passes ago has read its staging buffer, which is
+    // the one the epilogue warps fill after the next barrier.
+    if (OUT_MODE == kOutBf16) {
+      int useq = 0, sbuf = 0;
+      bool store_pending = false;
+      for (int u = blockIdx.x; u < p.total_units; u += gridDim.x, ++useq) {
+        const Unit w = decode_unit(p, u, TOK);
+        const CUtensorMap* tmap_y = w.lin == 0 ? &tmap_y0 : (w.lin == 1 ? &tmap_y1 : &tmap_y2);
+        named_bar_sync(1, kEpiBarThreads);                  // the unit's accumulator is complete (or the wait for it failed)
+        if (useq >= *epi_stop) break;
+        for (int pass = 0; pass < Plan::kPasses; ++pass, sbuf = (sbuf + 1 == Plan::kStagingBufs) ? 0 : sbuf + 1) {
+          const int tok_pass = w.tok0 + pass * Plan::kPassTok;
+          if (tok_pass >= p.M) break;
+          named_bar_sync(1, kEpiBarThreads);                // the pass is staged
+          if (lane == 0) {
+            tma_store_2d(tmap_y, base + Plan::kOffStaging + sbuf * Plan::kStagingBufBytes, w.n0, tok_pass);
+            bulk_commit_group();
+            bulk_wait_group_read<Plan::kStagingBufs - 2>();
+            store_pending = true;
+          }
+          __syncwarp();
+        }
+      }
+      if (lane == 0 && store_pending) bulk_wait_group0();
+    }
   } else {
     // ------------------------------------------------------------------ epilogue
     // TMEM lane = output feature, column = token.  Only the first epilogue warp polls the mbarrier;
     // the others are parked on a hardware barrier, which every epilogue warp reaches every time.
+    // bf16 tiles: the store warp takes part in these barriers too.
     const int ew = warp - kFirstEpiWarp;
     const int quad = warp & 3;                          // TMEM lane quadrant this warp may read
     const int colpart = ew >> 2;                        // 0 or 1: which 16-column chunks this warp takes
@@ -686,27 +726,25 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     const bool elected = (ew == 0 && lane == 0);
     constexpr int kChunksPerPass = Plan::kPassTok / 16;
     int useq = 0;
-    uint32_t passes_done = 0;                           // staging buffer = passes_done & 1
-    bool store_pending = false;
+    int sbuf = 0;                                       // staging buffer of the next pass
     for (int u = blockIdx.x; u < p.total_units; u += gridDim.x, ++useq) {
       const Unit w = decode_unit(p, u, TOK);
       const LinearDesc& L = p.lin[w.lin];
-      const CUtensorMap* tmap_y = w.lin == 0 ? &tmap_y0 : (w.lin == 1 ? &tmap_y1 : &tmap_y2);
       const int n = w.n0 + f;
       const float bias = (L.bias != nullptr && n < L.N && w.z == 0) ? L.bias[n] : 0.0f;
       if (ew == 0 && !mbar_wait(bar_acc_full, (uint32_t)useq & 1u, abort_flag)) {
         *epi_stop = useq;
         __threadfence_block();
       }
-      named_bar_sync(1, kNumEpiWarps * 32);
+      named_bar_sync(1, kEpiBarThreads);
       if (useq >= *epi_stop) { ok = false; break; }
       tcgen05_fence_after();
       if (OUT_MODE == kOutBf16) {
-        for (int pass = 0; pass < Plan::kPasses; ++pass, ++passes_done) {
+        for (int pass = 0; pass < Plan::kPasses; ++pass, sbuf = (sbuf + 1 == Plan::kStagingBufs) ? 0 : sbuf + 1) {
           const int tok_pass = w.tok0 + pass * Plan::kPassTok;
           if (tok_pass >= p.M) break;                       // uniform over the epilogue warps
           __nv_bfloat16* const buf = reinterpret_cast<__nv_bfloat16*>(smem + Plan::kOffStaging +
-                                                                       (passes_done & 1u) * Plan::kStagingBufBytes);
+                                                                       sbuf * Plan::kStagingBufBytes);
           for (int c = colpart; c < kChunksPerPass; c += 2) {
             uint32_t v[16];
             tmem_ld16(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)(pass * Plan::kPassTok + c * 16), v);
@@ -715,15 +753,8 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
               buf[(c * 16 + j) * kTileN + f] = __float2bfloat16_rn(__uint_as_float(v[j]) + bias);
           }
           fence_proxy_async_smem();                         // staged rows visible to the TMA store
-          // the store of the previous pass has read the other buffer, which the next pass will fill
-          if (elected && store_pending) bulk_wait_group_read0();
           if (pass == Plan::kPasses - 1 || tok_pass + Plan::kPassTok >= p.M) tcgen05_fence_before();
-          named_bar_sync(1, kNumEpiWarps * 32);
-          if (elected) {
-            tma_store_2d(tmap_y, smem_u32(buf), w.n0, tok_pass);
-            bulk_commit_group();
-            store_pending = true;
-          }
+          named_bar_sync(1, kEpiBarThreads);                // the store warp issues the pass's store
         }
       } else {
         constexpr int kChunks = TOK / 16;
@@ -741,12 +772,11 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
           }
         }
         tcgen05_fence_before();
-        named_bar_sync(1, kNumEpiWarps * 32);
+        named_bar_sync(1, kEpiBarThreads);
       }
       // accumulator drained: the MMA warp may start the next unit
       if (elected) mbar_arrive(bar_acc_empty);
     }
-    if (elected && store_pending) bulk_wait_group0();
     if (!ok) *abort_flag = 1;
   }
 
