@@ -160,6 +160,10 @@ __device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity,
 __device__ __forceinline__ void named_bar_sync(uint32_t id, uint32_t nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
+// Signs a hardware barrier without waiting for it (producer side of a producer / consumer pair).
+__device__ __forceinline__ void named_bar_arrive(uint32_t id, uint32_t nthreads) {
+  asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
@@ -438,8 +442,9 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
   const uint32_t tmem_d = *tmem_slot;
 
   bool ok = true;
-  // threads at the epilogue's hardware barrier: for bf16 tiles the store warp takes part
+  // threads at the epilogue's hardware barriers: for bf16 tiles the store warp takes part
   constexpr int kEpiBarThreads = (kNumEpiWarps + (OUT_MODE == kOutBf16 ? 1 : 0)) * 32;
+  constexpr uint32_t kBarUnit = 1, kBarStaged = 2, kBarFree = 3, kBarDrained = 4;
 
   if (warp == 0 || warp == kAProducerWarp) {
     // ------------------------------------------------------------------ TMA producers
@@ -686,27 +691,39 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     }
   } else if (warp == kStoreWarp) {
     // ------------------------------------------------------------------ store warp (bf16 tiles)
-    // Walks the units and passes like the epilogue warps and meets them at their hardware barrier:
-    // once a pass is staged, one lane issues its TMA store, so that issuing the store (some hundred
-    // cycles) is off the path of the warps that drain the accumulator.  Before it comes back to the
-    // barrier it waits until the store issued two passes ago has read its staging buffer, which is
-    // the one the epilogue warps fill after the next barrier.
+    // Walks the units and passes like the epilogue warps.  Two hardware barriers connect them in the
+    // producer / consumer way: the epilogue warps sign "staged" (bar.arrive) when a pass sits in its
+    // staging buffer and this warp waits for it (bar.sync); this warp signs "free" when the staging
+    // buffer of a pass may be written and the epilogue warps wait for that.  Neither side waits for the
+    // other's work: "free" for the next pass is signed before the store of this pass is issued (its
+    // buffer was last read by the store issued two passes ago), so issuing a store, some hundred cycles,
+    // runs beside the draining of the next pass.
     if (OUT_MODE == kOutBf16) {
       int useq = 0, sbuf = 0;
-      bool store_pending = false;
+      bool store_pending = false, first = true;
       for (int u = blockIdx.x; u < p.total_units; u += gridDim.x, ++useq) {
         const Unit w = decode_unit(p, u, TOK);
         const CUtensorMap* tmap_y = w.lin == 0 ? &tmap_y0 : (w.lin == 1 ? &tmap_y1 : &tmap_y2);
-        named_bar_sync(1, kEpiBarThreads);                  // the unit's accumulator is complete (or the wait for it failed)
+        named_bar_sync(kBarUnit, kEpiBarThreads);           // the unit's accumulator is complete (or the wait for it failed)
         if (useq >= *epi_stop) break;
         for (int pass = 0; pass < Plan::kPasses; ++pass, sbuf = (sbuf + 1 == Plan::kStagingBufs) ? 0 : sbuf + 1) {
           const int tok_pass = w.tok0 + pass * Plan::kPassTok;
           if (tok_pass >= p.M) break;
-          named_bar_sync(1, kEpiBarThreads);                // the pass is staged
+          if (first) {                                      // all staging buffers start free
+            named_bar_arrive(kBarFree, kEpiBarThreads);
+            first = false;
+          }
+          named_bar_sync(kBarStaged, kEpiBarThreads);       // the pass is staged
+          const bool more = (pass + 1 < Plan::kPasses && tok_pass + Plan::kPassTok < p.M) || u + (int)gridDim.x < p.total_units;
+          if (more) {
+            // the next pass's buffer was last read by the store issued two passes ago
+            if (lane == 0 && store_pending) bulk_wait_group_read<Plan::kStagingBufs - 2>();
+            __syncwarp();
+            named_bar_arrive(kBarFree, kEpiBarThreads);
+          }
           if (lane == 0) {
             tma_store_2d(tmap_y, base + Plan::kOffStaging + sbuf * Plan::kStagingBufBytes, w.n0, tok_pass);
             bulk_commit_group();
-            bulk_wait_group_read<Plan::kStagingBufs - 2>();
             store_pending = true;
           }
           __syncwarp();
@@ -736,7 +753,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         *epi_stop = useq;
         __threadfence_block();
       }
-      named_bar_sync(1, kEpiBarThreads);
+      named_bar_sync(kBarUnit, kEpiBarThreads);
       if (useq >= *epi_stop) { ok = false; break; }
       tcgen05_fence_after();
       if (OUT_MODE == kOutBf16) {
@@ -745,17 +762,26 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
           if (tok_pass >= p.M) break;                       // uniform over the epilogue warps
           __nv_bfloat16* const buf = reinterpret_cast<__nv_bfloat16*>(smem + Plan::kOffStaging +
                                                                        sbuf * Plan::kStagingBufBytes);
-          for (int c = colpart; c < kChunksPerPass; c += 2) {
+          // at most one 16-column chunk per warp and pass (kPassTok <= 32, two warps per lane quadrant)
+          static_assert(kChunksPerPass <= 2, "one chunk per warp and pass");
+          const bool mine = colpart < kChunksPerPass;
+          __nv_bfloat16 h[16];
+          if (mine) {
             uint32_t v[16];
-            tmem_ld16(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)(pass * Plan::kPassTok + c * 16), v);
+            tmem_ld16(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)(pass * Plan::kPassTok + colpart * 16), v);
 #pragma unroll
-            for (int j = 0; j < 16; ++j)
-              buf[(c * 16 + j) * kTileN + f] = __float2bfloat16_rn(__uint_as_float(v[j]) + bias);
+            for (int j = 0; j < 16; ++j) h[j] = __float2bfloat16_rn(__uint_as_float(v[j]) + bias);
+          }
+          if (pass == Plan::kPasses - 1 || tok_pass + Plan::kPassTok >= p.M) tcgen05_fence_before();
+          named_bar_sync(kBarFree, kEpiBarThreads);         // the staging buffer of this pass may be written
+          if (mine) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) buf[(colpart * 16 + j) * kTileN + f] = h[j];
           }
           fence_proxy_async_smem();                         // staged rows visible to the TMA store
-          if (pass == Plan::kPasses - 1 || tok_pass + Plan::kPassTok >= p.M) tcgen05_fence_before();
-          named_bar_sync(1, kEpiBarThreads);                // the store warp issues the pass's store
+          named_bar_arrive(kBarStaged, kEpiBarThreads);     // the store warp issues the pass's store
         }
+        named_bar_sync(kBarDrained, kNumEpiWarps * 32);     // every epilogue warp has read its part of the accumulator
       } else {
         constexpr int kChunks = TOK / 16;
         for (int c = colpart; c < kChunks; c += 2) {
@@ -772,7 +798,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
           }
         }
         tcgen05_fence_before();
-        named_bar_sync(1, kEpiBarThreads);
+        named_bar_sync(kBarDrained, kNumEpiWarps * 32);
       }
       // accumulator drained: the MMA warp may start the next unit
       if (elected) mbar_arrive(bar_acc_empty);
