@@ -870,13 +870,15 @@ int pick_tok_tile(int M) {
   return 256;
 }
 
+// SMs of the current device (cached per device id).
 int sm_count() {
-  static int n = 0;
+  static std::atomic<int> cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  int n = cached[dev].load();
   if (n == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-      n = 0;
-    if (n <= 0) n = 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cached[dev].store(n);
   }
   return n;
 }
@@ -886,11 +888,9 @@ int launch_one(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorMap* 
                cudaStream_t st) {
   using Plan = SmemPlan<TOK, DEQUANT, OUT_MODE>;
   auto kern = w4a16_gemm_kernel<TOK, DEQUANT, OUT_MODE>;
-  static bool configured = false;           // per instantiation
-  if (!configured) {
+  static std::atomic<unsigned long long> configured{0};      // per instantiation, one bit per device
+  if (first_use_on_device(configured))
     QZO_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Plan::kDynamicBytes));
-    configured = true;
-  }
   const int grid = p.total_units < sm_count() ? p.total_units : sm_count();
   QZO_LAUNCH(kern, dim3(grid), dim3(kThreads), Plan::kDynamicBytes, st, tx, tw, ty[0], ty[1], ty[2], p);
   return QZO_OK;

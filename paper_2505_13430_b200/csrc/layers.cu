@@ -493,13 +493,15 @@ int launch_attention(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_
   if ((ldq % 8) || (ldk % 8) || (ldv % 8) || (ldo % 2)) return QZO_ERR_BAD_ARG;
   if (dh == 64) {
     constexpr int smem = (kAttBQ + 4 * kAttBK) * (64 + 8) * 2;
-    static bool cfg = false;
-    if (!cfg) { QZO_CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)); cfg = true; }
+    static std::atomic<unsigned long long> cfg{0};
+    if (first_use_on_device(cfg))
+      QZO_CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     QZO_LAUNCH(attention_mma_kernel<64>, grid, dim3(kAttThreads), smem, st, q, k, v, ldq, ldk, ldv, out, ldo, S, scale_log2e);
   } else if (dh == 128) {
     constexpr int smem = (kAttBQ + 4 * kAttBK) * (128 + 8) * 2;
-    static bool cfg = false;
-    if (!cfg) { QZO_CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)); cfg = true; }
+    static std::atomic<unsigned long long> cfg{0};
+    if (first_use_on_device(cfg))
+      QZO_CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     QZO_LAUNCH(attention_mma_kernel<128>, grid, dim3(kAttThreads), smem, st, q, k, v, ldq, ldk, ldv, out, ldo, S, scale_log2e);
   } else {
     return QZO_ERR_BAD_ARG;

@@ -5,6 +5,7 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 #include <stddef.h>
+#include <atomic>
 
 #include "../../include/qzo.h"
 
@@ -32,6 +33,16 @@ constexpr int kGroup = 128;          // rows of one quantisation group (paper: g
 constexpr int kTileN = 128;          // output features per GEMM tile (UMMA M)
 constexpr int kBlockK = 64;          // K elements per pipeline stage (one 128-byte swizzle atom of bf16)
 constexpr int kPackedTileBytes = kTileN * kBlockK / 2;   // 4096: one (n-tile, k-block) of packed nibbles
+
+// True the first time it is called for the current device with this mask (one bit per device id
+// below 64; beyond that always true): per-device set-up such as cudaFuncSetAttribute is done once on
+// every device a process uses, not once per process.
+inline bool first_use_on_device(std::atomic<unsigned long long>& mask) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;
+  const unsigned long long bit = 1ull << dev;
+  return (mask.fetch_or(bit) & bit) == 0;
+}
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
