@@ -162,3 +162,27 @@ def test_empty_and_minimal_calls(lib):
     ref = omodel.forward_loss(om, t1.cpu().numpy(), l1.cpu().numpy(), 3, +1, 1e-3)
     assert abs(loss - ref) <= 1e-3
     gm.close()
+
+
+@pytest.mark.parametrize("name", ["tiny", "tiny_opt"])
+def test_step_in_one_pass_equals_two_separate_passes(lib, name):
+    # With 256 tokens the step runs both perturbation signs as one forward over two copies of the
+    # batch; with 192 tokens (no token-tile boundary between the copies) it runs two forwards.  Either
+    # way the losses it reports are, bit for bit, those of the single-sign entry point, and they match
+    # the oracle.
+    cfg, c, om, gm, tok, lab = _setup(lib, name)
+    seed, eps = 17, c["eps"]
+    for rows in (c["batch"], c["batch"] - 1):
+        t, l = tok[:rows].contiguous(), lab[:rows].contiguous()
+        t_d, l_d = t.cuda(), l.cuda()
+        lp = gm.qzo_forward_loss(t_d, l_d, seed, +1, eps).cpu().clone()
+        lm = gm.qzo_forward_loss(t_d, l_d, seed, -1, eps).cpu().clone()
+        before = gm.scales.clone()
+        out = gm.qzo_step(t_d, l_d, seed, eps, c["lr"], c["clip"])
+        gm.scales.copy_(before)
+        assert np.float32(out[0]) == np.float32(lp[0]) and np.float32(out[1]) == np.float32(lm[0]), rows
+        ref_p = omodel.forward_loss(om, t.numpy(), l.numpy(), seed, +1, eps)
+        ref_m = omodel.forward_loss(om, t.numpy(), l.numpy(), seed, -1, eps)
+        assert abs(out[0] - ref_p) <= 1e-3 and abs(out[1] - ref_m) <= 1e-3, rows
+    assert gm.qzo_device_status() == 0
+    gm.close()
