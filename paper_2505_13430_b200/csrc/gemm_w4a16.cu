@@ -23,7 +23,8 @@
 //   warp 3       watch warp: does the mbarrier waits the issuer depends on and publishes a count
 //   warps 4-7    scale warps: Philox4x32-10 + Box-Muller, s' = s + sign eps z in fp32, split
 //                into bf16 hi + lo parts, written next to the nibbles of the group's A slot
-//   warps 8-15   de-quantisers: nibbles -> bf16 (u - 8) * s' written to the A stages in TMEM
+//   warps 8-15   de-quantisers: nibbles -> bf16 (u - 8) * s' written to the A stages in TMEM; two teams
+//                of four warps take alternate quantisation groups
 //   warps 16-23  epilogue: TMEM -> registers (+ bias) -> bf16 rows in shared memory, 32 tokens per pass
 //   warp 24      store warp: issues the TMA store of every staged pass (three staging buffers), so
 //                that the warps draining the single accumulator never wait for a store to be issued
@@ -428,7 +429,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     for (int s = 0; s < kASlots; ++s) {
       // int4 path: the slot is full when its nibbles have landed AND its perturbed scales are written
       mbar_init(bar_a_full(s), DEQUANT ? 2 : 1);
-      mbar_init(bar_a_deq(s), kNumDeqWarps);
+      mbar_init(bar_a_deq(s), kNumDeqWarps / 2);        // one team of four de-quantiser warps per group
       mbar_init(bar_a_empty(s), 1);
     }
     mbar_init(bar_acc_full, 1);
@@ -634,7 +635,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     if (DEQUANT) {
       const int dt = threadIdx.x - kFirstDeqWarp * 32;      // 0..255
       const int r = (warp & 3) * 32 + lane;                 // row of the tile = TMEM lane this warp may access
-      const int h = dt >> 7;                                // half of the k-block (32 k each)
+      const int team = dt >> 7;                             // two teams of four warps take alternate groups
       const __nv_bfloat162 magic_bias = __halves2bfloat162(__float2bfloat16_rn(136.0f), __float2bfloat16_rn(136.0f));
       __nv_bfloat162 s_hi, s_lo;
       *reinterpret_cast<uint32_t*>(&s_hi) = 0u;
@@ -654,37 +655,46 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         }
       };
       // A stage in tensor memory: lane = row (this warp's quadrant), column = k / 2
-      const uint32_t a_lane_base = tmem_d + ((uint32_t)((warp & 3) * 32) << 16) + kAccCols + (uint32_t)(h * 16);
-      Ring ra;                              // A-ring slot = one quantisation group (two k-blocks)
+      const uint32_t a_lane_base = tmem_d + ((uint32_t)((warp & 3) * 32) << 16) + kAccCols;
+      int gig = 0;                          // quantisation groups visited by this CTA so far (all units)
       for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x) {
         const Unit w = decode_unit(p, u, TOK);
-        for (int it = 0; it < w.nkb; it += 2) {
+        for (int it = 0; it < w.nkb; it += 2, ++gig) {
+          if ((gig & 1) != team) continue;                    // the other team's group
+          const int slot = gig % kASlots;                     // A-ring slot = one quantisation group (two k-blocks)
+          const uint32_t gph = (uint32_t)(gig / kASlots) & 1u;
           const bool two = it + 1 < w.nkb;                    // the last group of an odd K has one k-block
           // the slot is full: nibbles landed, perturbed scales written; that implies it had been released
           // by the MMAs that last read it
-          if (!__all_sync(0xffffffffu, mbar_wait(bar_a_full(ra.s), ra.ph, abort_flag))) { ok = false; break; }
+          if (!__all_sync(0xffffffffu, mbar_wait(bar_a_full(slot), gph, abort_flag))) { ok = false; break; }
           {
-            const uint2 c = *reinterpret_cast<const uint2*>(smem + Plan::kOffCooked + ra.s * kCookedScaleBytes + r * 8);
+            const uint2 c = *reinterpret_cast<const uint2*>(smem + Plan::kOffCooked + slot * kCookedScaleBytes + r * 8);
             *reinterpret_cast<uint32_t*>(&s_hi) = c.x;
             *reinterpret_cast<uint32_t*>(&s_lo) = c.y;
           }
-          const uint8_t* src = smem + Plan::kOffA + ra.s * (2 * Plan::kAStageBytes) + (h * kTileN + r) * 16;
-          const uint4 pk0 = *reinterpret_cast<const uint4*>(src);
-          uint4 pk1 = make_uint4(0, 0, 0, 0);
-          if (two) pk1 = *reinterpret_cast<const uint4*>(src + Plan::kAStageBytes);
+          // this row's 64 k of each k-block: two 16-byte units (32 k each)
+          const uint8_t* src = smem + Plan::kOffA + slot * (2 * Plan::kAStageBytes) + r * 16;
+          uint4 pk[4];
+          pk[0] = *reinterpret_cast<const uint4*>(src);
+          pk[1] = *reinterpret_cast<const uint4*>(src + kTileN * 16);
+          pk[2] = pk[3] = make_uint4(0, 0, 0, 0);
+          if (two) {
+            pk[2] = *reinterpret_cast<const uint4*>(src + Plan::kAStageBytes);
+            pk[3] = *reinterpret_cast<const uint4*>(src + Plan::kAStageBytes + kTileN * 16);
+          }
           tcgen05_fence_after();                              // orders the MMAs' reads of this slot before the stores below
           uint32_t outw[16];
-          dequant16(pk0, outw);
-          tmem_st16(a_lane_base + (uint32_t)((ra.s * 2) * kATmemColsPerStage), outw);
-          if (two) {
-            dequant16(pk1, outw);
-            tmem_st16(a_lane_base + (uint32_t)((ra.s * 2 + 1) * kATmemColsPerStage), outw);
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            if (q4 < 2 || two) {
+              dequant16(pk[q4], outw);
+              tmem_st16(a_lane_base + (uint32_t)((slot * 2 + (q4 >> 1)) * kATmemColsPerStage + (q4 & 1) * 16), outw);
+            }
           }
           tmem_wait_st();
           tcgen05_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(bar_a_deq(ra.s));
-          ra.next(kASlots);
+          if (lane == 0) mbar_arrive(bar_a_deq(slot));
         }
       }
       if (!ok) *abort_flag = 1;
