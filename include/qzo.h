@@ -214,7 +214,9 @@ int qzo_step_host(qzo_model* m, const int32_t* h_tokens, const int32_t* h_labels
 int qzo_debug_set_capture(qzo_model* m, int layer);
 /* Copies an intermediate of the LAST forward into d_out (bf16 [T][d] for which = 0: output of
  * decoder block `layer`, which must be the block chosen with qzo_debug_set_capture before that
- * forward; float [T][V] for which = 1: logits, layer ignored). */
+ * forward; float [T][V] for which = 1: logits, layer ignored).  T is the token count of that
+ * forward: B*S after qzo_forward_loss, 2*B*S after a qzo_step that ran both signs as one pass
+ * (rows of the sign +1 copy first).  bytes below the size needed: QZO_ERR_BAD_ARG. */
 int qzo_debug_layer_output(qzo_model* m, int layer, int which, void* d_out, size_t bytes);
 
 /* Reads the device status word (0 = no bounded wait has expired since init). Synchronises. */
