@@ -270,6 +270,11 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t v[16]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
 // Shared-memory matrix descriptor of a K-major bf16 tile with 128-byte swizzle: rows are
 // 128 bytes, eight rows form a 1024-byte swizzle atom (stride byte offset 1024), descriptor
 // version 1, layout type 2 (128-byte swizzle).  The tile base must be 1024-byte aligned; a
@@ -767,29 +772,62 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
       if (useq >= *epi_stop) { ok = false; break; }
       tcgen05_fence_after();
       if (OUT_MODE == kOutBf16) {
-        for (int pass = 0; pass < Plan::kPasses; ++pass, sbuf = (sbuf + 1 == Plan::kStagingBufs) ? 0 : sbuf + 1) {
-          const int tok_pass = w.tok0 + pass * Plan::kPassTok;
-          if (tok_pass >= p.M) break;                       // uniform over the epilogue warps
-          __nv_bfloat16* const buf = reinterpret_cast<__nv_bfloat16*>(smem + Plan::kOffStaging +
-                                                                       sbuf * Plan::kStagingBufBytes);
-          // at most one 16-column chunk per warp and pass (kPassTok <= 32, two warps per lane quadrant)
-          static_assert(kChunksPerPass <= 2, "one chunk per warp and pass");
-          const bool mine = colpart < kChunksPerPass;
-          __nv_bfloat16 h[16];
+        // at most one 16-column chunk per warp and pass (kPassTok <= 32, two warps per lane quadrant)
+        static_assert(kChunksPerPass <= 2, "one chunk per warp and pass");
+        const bool mine = colpart < kChunksPerPass;
+        // TMEM -> registers: this thread's feature for the 16 tokens of its chunk, as eight bf16 pairs
+        auto load_pass = [&](int pass, uint32_t (&h)[8]) {
           if (mine) {
             uint32_t v[16];
             tmem_ld16(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)(pass * Plan::kPassTok + colpart * 16), v);
 #pragma unroll
-            for (int j = 0; j < 16; ++j) h[j] = __float2bfloat16_rn(__uint_as_float(v[j]) + bias);
+            for (int j = 0; j < 8; ++j)
+              h[j] = pack_bf16x2(__uint_as_float(v[2 * j]) + bias, __uint_as_float(v[2 * j + 1]) + bias);
           }
-          if (pass == Plan::kPasses - 1 || tok_pass + Plan::kPassTok >= p.M) tcgen05_fence_before();
+        };
+        // registers -> staging buffer -> (store warp) TMA store
+        auto stage_pass = [&](const uint32_t (&h)[8]) {
+          unsigned short* const buf = reinterpret_cast<unsigned short*>(smem + Plan::kOffStaging +
+                                                                        sbuf * Plan::kStagingBufBytes);
           named_bar_sync(kBarFree, kEpiBarThreads);         // the staging buffer of this pass may be written
           if (mine) {
 #pragma unroll
-            for (int j = 0; j < 16; ++j) buf[(colpart * 16 + j) * kTileN + f] = h[j];
+            for (int j = 0; j < 8; ++j) {
+              buf[(colpart * 16 + 2 * j) * kTileN + f] = (unsigned short)(h[j] & 0xFFFFu);
+              buf[(colpart * 16 + 2 * j + 1) * kTileN + f] = (unsigned short)(h[j] >> 16);
+            }
           }
           fence_proxy_async_smem();                         // staged rows visible to the TMA store
           named_bar_arrive(kBarStaged, kEpiBarThreads);     // the store warp issues the pass's store
+          sbuf = (sbuf + 1 == Plan::kStagingBufs) ? 0 : sbuf + 1;
+        };
+        // A full tile of at least four passes: the last half of the passes is first only read into
+        // registers, so that the accumulator is handed back to the MMA warp before those passes are
+        // staged and stored (the accumulator is single, its drain time is taken from the tensor pipe).
+        constexpr int kHold = Plan::kPasses >= 4 ? Plan::kPasses / 2 : 0;
+        if (kHold > 0 && w.tok0 + TOK <= p.M) {
+          for (int pass = 0; pass < Plan::kPasses - kHold; ++pass) {
+            uint32_t h[8];
+            load_pass(pass, h);
+            stage_pass(h);
+          }
+          uint32_t held[kHold > 0 ? kHold : 1][8];
+#pragma unroll
+          for (int k = 0; k < kHold; ++k) load_pass(Plan::kPasses - kHold + k, held[k]);
+          tcgen05_fence_before();
+          named_bar_sync(kBarDrained, kNumEpiWarps * 32);   // every epilogue warp has read its part of the accumulator
+          if (elected) mbar_arrive(bar_acc_empty);          // the MMA warp may start the next unit
+#pragma unroll
+          for (int k = 0; k < kHold; ++k) stage_pass(held[k]);
+          continue;
+        }
+        for (int pass = 0; pass < Plan::kPasses; ++pass) {
+          const int tok_pass = w.tok0 + pass * Plan::kPassTok;
+          if (tok_pass >= p.M) break;                       // uniform over the epilogue warps
+          uint32_t h[8];
+          load_pass(pass, h);
+          if (pass == Plan::kPasses - 1 || tok_pass + Plan::kPassTok >= p.M) tcgen05_fence_before();
+          stage_pass(h);
         }
         named_bar_sync(kBarDrained, kNumEpiWarps * 32);     // every epilogue warp has read its part of the accumulator
       } else {
