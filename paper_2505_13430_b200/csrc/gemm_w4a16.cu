@@ -26,6 +26,7 @@
 //   warps 8-15   de-quantisers: nibbles -> bf16 (u - 8) * s' written to the A stages in TMEM; two teams
 //                of four warps take alternate quantisation groups
 //   warps 16-23  epilogue: TMEM -> registers (+ bias) -> bf16 rows in shared memory, 32 tokens per pass
+//                (the last passes of a full tile wait in registers: the accumulator is released first)
 //   warp 24      store warp: issues the TMA store of every staged pass (three staging buffers), so
 //                that the warps draining the single accumulator never wait for a store to be issued
 // Every wait on an mbarrier is bounded; when a wait expires the CTA records an error in
