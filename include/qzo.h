@@ -47,7 +47,7 @@ typedef enum {
   QZO_ERR_UNSUPPORTED_DEVICE = -2, /* current device is not sm_100 */
   QZO_ERR_WORKSPACE = -3,          /* workspace too small or misaligned (256 bytes) */
   QZO_ERR_NONFINITE = -4,          /* a loss or g is NaN/Inf; scales were left untouched */
-  QZO_ERR_DEVICE_TIMEOUT = -5,     /* a bounded device-side wait expired (status word) */
+  QZO_ERR_DEVICE_TIMEOUT = -5,     /* a bounded device-side wait expired (status word); scales untouched by that step */
   QZO_ERR_CUDA = -6,               /* a CUDA call failed; see qzo_last_cuda_error */
   QZO_ERR_MISSING_TENSOR = -7      /* qzo_init_model: a required tensor was not supplied */
 } qzo_status;
@@ -119,7 +119,9 @@ int qzo_perturbed_gemm(const void* d_x_bf16, const void* d_wq, const void* d_sca
  *  - A problem whose partial sums (qzo_gemm_workspace_bytes) exceed the array returns
  *    QZO_ERR_WORKSPACE and launches nothing.
  *  - The first call on each device looks the array's device address up (with that device
- *    current); make that first call before any stream capture begins.
+ *    current).  If no kernel of the library has run on that device yet, this is also the moment the
+ *    driver loads the library's device code and reserves the array, which may synchronise the device:
+ *    make that first call at start-up, and before any stream capture begins.  Later calls do neither.
  *  - All calls on a device share the one array, which keeps the last call's partial sums (none
  *    of it needs clearing: each call overwrites every element it later reads).  Two calls that
  *    overlap on the GPU (different streams) race on it; keep them on one stream or order them. */
@@ -200,15 +202,44 @@ int qzo_update_scales(qzo_model* m, uint64_t seed, float lr, float g, float clip
  * -eps z); every kernel works row by row or sequence by sequence, so the losses are the ones two
  * separate passes give, bit for bit, when both use the same token tile (B*S >= 256).
  * h_out (may be NULL): {l+, l-, d, d'}; when
- * non-NULL the call synchronises the stream.  If either loss is not finite the scales are
- * left untouched and (when h_out is given) QZO_ERR_NONFINITE is returned. */
+ * non-NULL the call synchronises the stream.  The scales are left untouched (the update coefficient is
+ * forced to zero on the device) and, when h_out is given, an error is returned if
+ *  - either loss is not finite: QZO_ERR_NONFINITE;
+ *  - a bounded device-side wait expired in any launch since qzo_init_model: QZO_ERR_DEVICE_TIMEOUT;
+ *  - a token id lies outside [0, vocab): QZO_ERR_BAD_ARG.
+ * The last two are sticky (status word, see qzo_device_status). */
 int qzo_step(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S,
              uint64_t seed, float eps, float lr, float clip, float* h_out);
+
+/* The two halves of qzo_step, for data-parallel replicas (every rank holds the same theta_bar and Delta
+ * and its own part of the batch; z depends on (seed, index) only, Sec. 3.1, so ranks exchange losses,
+ * never parameters).
+ * qzo_step_begin runs the two forward passes of Algorithm 1 on this rank's tokens and writes
+ *   d_sums (device, float[4], 16-byte aligned) = {sum of token losses with +eps z, the same with -eps z,
+ *   kept tokens of the + pass, kept tokens of the - pass}.
+ * Between the calls the caller may add the d_sums of all ranks element by element (one all-reduce of four
+ * floats, asynchronously on the same stream).  qzo_step_finish then forms l+- = sum / count, d = (l+ - l-) /
+ * (2 eps), d' = clip(d, -C, C) (Eq. 6) and applies the seeded update (Algorithm 1, last loop), all on the
+ * device; given equal d_sums and seed every rank ends with bit-identical scales.  h_out and the error
+ * behaviour are those of qzo_step.  qzo_step is qzo_step_begin followed by qzo_step_finish. */
+int qzo_step_begin(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S,
+                   uint64_t seed, float eps, float* d_sums);
+int qzo_step_finish(qzo_model* m, const float* d_sums, uint64_t seed, float eps, float lr, float clip,
+                    float* h_out);
 
 /* Same step with HOST token / label buffers (int32 [B][S]); copies them in, runs the step and
  * reads {l+, l-, d, d'} back.  Synchronises. */
 int qzo_step_host(qzo_model* m, const int32_t* h_tokens, const int32_t* h_labels, int B, int S,
                   uint64_t seed, float eps, float lr, float clip, float* h_out);
+
+/* The trainable state (Algorithm 1 "Require": the quantisation scales Delta that the caller hands over
+ * and gets back).  linear_id = layer * L + position, L = 7 (Llama: q,k,v,o,gate,up,down) or 6 (OPT:
+ * q,k,v,o,fc1,fc2): copies that linear's bf16 [G][N] scales out of / into the model's flat buffer;
+ * linear_id = -1: the whole flat buffer (qzo_num_scales entries).  d_bf16 is a device pointer; `bytes` must
+ * be exactly the size of what is copied (QZO_ERR_BAD_ARG otherwise).  Asynchronous on the model's stream.
+ * Because z is a function of (seed, index) only, scales + step counter + base seed resume a run exactly. */
+int qzo_get_scales(qzo_model* m, int linear_id, void* d_bf16, size_t bytes);
+int qzo_set_scales(qzo_model* m, int linear_id, const void* d_bf16, size_t bytes);
 
 /* Selects the decoder block whose output later forwards keep a copy of (-1 = none). */
 int qzo_debug_set_capture(qzo_model* m, int layer);
@@ -219,8 +250,13 @@ int qzo_debug_set_capture(qzo_model* m, int layer);
  * (rows of the sign +1 copy first).  bytes below the size needed: QZO_ERR_BAD_ARG. */
 int qzo_debug_layer_output(qzo_model* m, int layer, int which, void* d_out, size_t bytes);
 
-/* Reads the device status word (0 = no bounded wait has expired since init). Synchronises. */
+/* Reads the device status word: bit 0 = a bounded device-side wait expired in some launch since init
+ * (returns QZO_ERR_DEVICE_TIMEOUT), bit 1 = a token id outside [0, vocab) was seen (QZO_ERR_BAD_ARG);
+ * 0 = nothing to report.  Synchronises. */
 int qzo_device_status(qzo_model* m, int* h_status);
+/* Overwrites the status word from the host (0 clears it).  For tests of the error path of a step and
+ * for clearing the word after the caller has dealt with a report.  Synchronises. */
+int qzo_debug_set_status(qzo_model* m, int value);
 
 /* Per-GEMM timing: with max_launches > 0 every later perturbed-GEMM launch of this model (up to
  * max_launches between two reads) is bracketed by a pair of CUDA events on the model's stream;

@@ -9,7 +9,7 @@ LIB = os.path.join(HERE, "libqzo.so")
 SOURCES = ["prims.cu", "gemm_w4a16.cu", "layers.cu", "model.cu"]
 HEADERS = ["qzo_common.cuh", "philox.cuh", "launch.cuh", "layers.cuh", os.path.join("..", "..", "include", "qzo.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-Xcompiler", "-fPIC", "--use_fast_math=false"]
+              "-Xcompiler", "-fPIC"]
 
 
 def _stale():
@@ -25,7 +25,7 @@ def build(force=False, verbose=False):
     if not force and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    flags = [f for f in NVCC_FLAGS if not f.startswith("--use_fast_math")]
+    flags = list(NVCC_FLAGS)
     if verbose:
         flags += ["-Xptxas", "-v"]
     objs = []

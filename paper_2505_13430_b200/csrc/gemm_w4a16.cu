@@ -855,7 +855,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     if (!ok) *abort_flag = 1;
   }
 
-  if (!ok && p.status != nullptr) atomicExch(p.status, 1);
+  if (!ok && p.status != nullptr) atomicOr(p.status, kStatusTimeout);
   tcgen05_fence_before();
   __syncthreads();
   if (warp == 1) {
@@ -969,7 +969,7 @@ int gemm_splits(int M, int K, int N) {
   if (tok > 128) return 1;                       // 256-token tiles: plenty of units, tensor-bound
   const int tiles = ceil_div(N, kTileN) * ceil_div(M, tok);
   const int groups = ceil_div(K, kGroup);
-  const int sms = 148;
+  const int sms = sm_count();                    // of the current device (148 on B200)
   const double cycles_per_kb = 600.0, fill_cycles = 3500.0, clock_ghz = 1.8;
   int best = 1;
   double best_us = 1e30;

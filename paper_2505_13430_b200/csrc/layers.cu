@@ -42,11 +42,15 @@ __device__ __forceinline__ float block_max(float v, float* red) {
 }
 
 // x[t][:] = E[tok[t]][:] (+ P[t % S][:])
+// A token id outside [0, vocab) sets bit 1 of the status word (the step then reports a bad argument and
+// leaves the scales alone); the row is still written, from the nearest valid id, so nothing is read
+// out of bounds.
 __global__ void embedding_kernel(const int32_t* __restrict__ tokens, const __nv_bfloat16* __restrict__ embed,
                                  const __nv_bfloat16* __restrict__ pos, int S, int d, int vocab,
-                                 __nv_bfloat16* __restrict__ x) {
+                                 __nv_bfloat16* __restrict__ x, int* __restrict__ status) {
   const int t = blockIdx.x;
   int tok = tokens[t];
+  if ((tok < 0 || tok >= vocab) && threadIdx.x == 0 && status != nullptr) atomicOr(status, kStatusBadToken);
   tok = min(max(tok, 0), vocab - 1);
   const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(embed + (size_t)tok * d);
   const __nv_bfloat162* pp = pos ? reinterpret_cast<const __nv_bfloat162*>(pos + (size_t)(t % S) * d) : nullptr;
@@ -429,9 +433,10 @@ ce_rows_kernel(const float* __restrict__ logits, const int32_t* __restrict__ lab
   if (threadIdx.x == 0) row_loss[t] = (gmx + logf(total)) - row[label];
 }
 
-// loss = sum(row_loss over kept rows) / count, summed in a fixed order by one block.
+// loss = sum(row_loss over kept rows) / count, summed in a fixed order by one block; the sum and the
+// count are also written (sum_out, count_out may be null): they are what data-parallel ranks exchange.
 __global__ void ce_mean_kernel(const float* __restrict__ row_loss, const int32_t* __restrict__ labels, int T, int V,
-                               float* __restrict__ loss) {
+                               float* __restrict__ loss, float* __restrict__ sum_out, float* __restrict__ count_out) {
   __shared__ float red[32];
   float s = 0.0f, c = 0.0f;
   for (int i = threadIdx.x; i < T; i += blockDim.x) {
@@ -440,26 +445,34 @@ __global__ void ce_mean_kernel(const float* __restrict__ row_loss, const int32_t
   }
   s = block_sum(s, red);
   c = block_sum(c, red);
-  if (threadIdx.x == 0) *loss = s / fmaxf(c, 1.0f);
+  if (threadIdx.x == 0) {
+    if (loss) *loss = s / fmaxf(c, 1.0f);
+    if (sum_out) *sum_out = s;
+    if (count_out) *count_out = c;
+  }
 }
 
-// d = (l+ - l-) / (2 eps); d' = clip(d, -C, C) (Eq. 6); coef = lr * d' (0 if a loss is not finite).
-// out = {l+, l-, d, d', coef}
-__global__ void ddc_kernel(const float* __restrict__ lp, const float* __restrict__ lm, float eps, float lr, float clip,
+// sums = {sum of token losses with +eps z, the same with -eps z, kept tokens of each pass}:
+// l+- = sum / count; d = (l+ - l-) / (2 eps); d' = clip(d, -C, C) (Eq. 6); coef = lr * d', forced to 0
+// (no update) when a loss is not finite or the status word reports a failed launch or a bad token.
+// out = {l+, l-, d, d', coef, status word as a float}
+__global__ void ddc_kernel(const float* __restrict__ sums, float eps, float lr, float clip, const int* __restrict__ status,
                            float* __restrict__ out) {
-  const float a = *lp, b = *lm;
+  const float a = sums[0] / fmaxf(sums[2], 1.0f), b = sums[1] / fmaxf(sums[3], 1.0f);
   const float d = (a - b) / (2.0f * eps);
   const float dc = fminf(fmaxf(d, -clip), clip);
-  const bool finite = isfinite(a) && isfinite(b);
+  const int st = status ? *status : 0;
+  const bool good = isfinite(a) && isfinite(b) && st == 0;
   out[0] = a; out[1] = b; out[2] = d; out[3] = dc;
-  out[4] = finite ? __fmul_rn(lr, dc) : 0.0f;
+  out[4] = good ? __fmul_rn(lr, dc) : 0.0f;
+  out[5] = (float)st;
 }
 
 }  // namespace
 
 int launch_embedding(const int32_t* tokens, const __nv_bfloat16* embed, const __nv_bfloat16* pos, int T, int S, int d,
-                     int vocab, __nv_bfloat16* x, cudaStream_t st) {
-  QZO_LAUNCH(embedding_kernel, dim3(T), dim3(128), 0, st, tokens, embed, pos, S, d, vocab, x);
+                     int vocab, __nv_bfloat16* x, int* status, cudaStream_t st) {
+  QZO_LAUNCH(embedding_kernel, dim3(T), dim3(128), 0, st, tokens, embed, pos, S, d, vocab, x, status);
   return QZO_OK;
 }
 int launch_add_rmsnorm(__nv_bfloat16* x, const __nv_bfloat16* delta, const float* w, float eps, int T, int d,
@@ -519,13 +532,13 @@ int launch_relu(__nv_bfloat16* x, int64_t n, cudaStream_t st) {
   return QZO_OK;
 }
 int launch_cross_entropy(const float* logits, const int32_t* labels, int T, int V, float* row_loss, float* loss,
-                         cudaStream_t st) {
+                         float* sum_out, float* count_out, cudaStream_t st) {
   QZO_LAUNCH(ce_rows_kernel, dim3(T), dim3(256), 0, st, logits, labels, V, row_loss);
-  QZO_LAUNCH(ce_mean_kernel, dim3(1), dim3(1024), 0, st, row_loss, labels, T, V, loss);
+  QZO_LAUNCH(ce_mean_kernel, dim3(1), dim3(1024), 0, st, row_loss, labels, T, V, loss, sum_out, count_out);
   return QZO_OK;
 }
-int launch_ddc(const float* lp, const float* lm, float eps, float lr, float clip, float* out5, cudaStream_t st) {
-  QZO_LAUNCH(ddc_kernel, dim3(1), dim3(1), 0, st, lp, lm, eps, lr, clip, out5);
+int launch_ddc(const float* sums4, float eps, float lr, float clip, const int* status, float* out6, cudaStream_t st) {
+  QZO_LAUNCH(ddc_kernel, dim3(1), dim3(1), 0, st, sums4, eps, lr, clip, status, out6);
   return QZO_OK;
 }
 

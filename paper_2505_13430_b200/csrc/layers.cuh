@@ -4,7 +4,7 @@
 
 namespace qzo {
 int launch_embedding(const int32_t* tokens, const __nv_bfloat16* embed, const __nv_bfloat16* pos, int T, int S, int d,
-                     int vocab, __nv_bfloat16* x, cudaStream_t st);
+                     int vocab, __nv_bfloat16* x, int* status, cudaStream_t st);
 // x <- x + delta (skipped when delta is null), then y = norm(x); y may alias delta.
 int launch_add_rmsnorm(__nv_bfloat16* x, const __nv_bfloat16* delta, const float* w, float eps, int T, int d,
                        __nv_bfloat16* y, cudaStream_t st);
@@ -17,11 +17,14 @@ int launch_attention(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_
                      __nv_bfloat16* out, int ldo, int B, int S, int H, int dh, cudaStream_t st);
 int launch_silu_mul(const __nv_bfloat16* gate, const __nv_bfloat16* up, __nv_bfloat16* out, int64_t n, cudaStream_t st);
 int launch_relu(__nv_bfloat16* x, int64_t n, cudaStream_t st);
+// loss (mean), sum_out and count_out may each be null
 int launch_cross_entropy(const float* logits, const int32_t* labels, int T, int V, float* row_loss, float* loss,
-                         cudaStream_t st);
-int launch_ddc(const float* lp, const float* lm, float eps, float lr, float clip, float* out5, cudaStream_t st);
+                         float* sum_out, float* count_out, cudaStream_t st);
+// sums4 = {sum l+, sum l-, kept tokens (+), kept tokens (-)}; out6 = {l+, l-, d, d', lr d' or 0, status}
+int launch_ddc(const float* sums4, float eps, float lr, float clip, const int* status, float* out6, cudaStream_t st);
 
 // gemm_w4a16.cu
+constexpr int kMaxSplitTokens = 128;   // launches with more tokens never split along K
 int gemm_splits(int M, int K, int N);
 size_t gemm_workspace_bytes(int M, int K, int N);
 // One linear of a grouped launch: Y = X W' (+ bias), Y bf16 [M][ldo].

@@ -110,7 +110,7 @@ struct qzo_model {
   // workspace regions
   __nv_bfloat16 *x = nullptr, *xn = nullptr, *qkv = nullptr, *att = nullptr, *mlp_a = nullptr, *mlp_b = nullptr,
                 *capture = nullptr;
-  float *logits = nullptr, *row_loss = nullptr, *loss2 = nullptr, *out5 = nullptr, *rope_cs = nullptr;
+  float *logits = nullptr, *row_loss = nullptr, *loss2 = nullptr, *sums = nullptr, *out6 = nullptr, *rope_cs = nullptr;
   int32_t *tok_dev = nullptr, *lab_dev = nullptr;
   void* gemm_ws = nullptr;
   size_t gemm_ws_bytes = 0;
@@ -159,9 +159,14 @@ int plan_workspace(const qzo_model_desc& d, int max_tokens, WsPlan* p) {
   p->off_rope = take((size_t)d.max_seq * (dm / d.n_heads) * 4);
   p->off_tok = take((size_t)T * 4);
   p->off_lab = take((size_t)T * 4);
+  // split-K partial sums: the largest need over every token count a launch of this model can have
+  // (any B*S up to max_tokens in a single-sign pass, twice that in a paired step); only token counts
+  // up to the largest split token tile can split, the rest is covered by the two limits themselves
   size_t gb = 0;
-  for (int i = 0; i < nl; ++i)
+  for (int i = 0; i < nl; ++i) {
+    for (int M = 1; M <= std::min(T, kMaxSplitTokens); ++M) gb = std::max(gb, gemm_workspace_bytes(M, ls[i].K, ls[i].N));
     gb = std::max(gb, std::max(gemm_workspace_bytes(T, ls[i].K, ls[i].N), gemm_workspace_bytes(max_tokens, ls[i].K, ls[i].N)));
+  }
   p->gemm_bytes = gb;
   p->off_gemm = take(gb);
   p->total = off;
@@ -209,8 +214,10 @@ static int linear(qzo_model* m, const Linear& L, const __nv_bfloat16* in, __nv_b
 // is run with sign * eps, the second with -sign * eps, and d_loss[0], d_loss[1] receive the two mean
 // losses.  Every kernel works row by row or sequence by sequence, so each half computes exactly what
 // a pass of its own would.
+// d_loss (mean, may be null) and d_sums (may be null) receive the result: single pass: d_loss[0], d_sums[0] = sum of
+// token losses, d_sums[2] = kept tokens; paired: d_loss[0..1], d_sums[0..1] sums, d_sums[2..3] counts.
 int forward_loss(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S, uint64_t seed, int sign,
-                 float eps, float* d_loss, bool paired) {
+                 float eps, float* d_loss, float* d_sums, bool paired, int slot = 0) {
   const qzo_model_desc& d = m->desc;
   const int dm = d.d_model, H = d.n_heads, dh = dm / H, F = d.d_ffn;
   const int pair_rows = paired ? B * S : 0;
@@ -218,7 +225,7 @@ int forward_loss(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels,
   const int T = B * S;
   cudaStream_t st = m->stream;
   const bool llama = d.arch == QZO_ARCH_LLAMA;
-  QZO_TRY(launch_embedding(d_tokens, m->embed, llama ? nullptr : m->pos_embed, T, S, dm, d.vocab, m->x, st));
+  QZO_TRY(launch_embedding(d_tokens, m->embed, llama ? nullptr : m->pos_embed, T, S, dm, d.vocab, m->x, m->status, st));
   // The residual stream x is updated lazily: a projection writes its output to xn, and the norm that
   // follows adds it to x before normalising (x += xn; xn = norm(x)).
   const __nv_bfloat16* pending = nullptr;          // projection output not yet added to x
@@ -255,11 +262,12 @@ int forward_loss(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels,
   QZO_TRY(launch_bf16_gemm_f32out(m->xn, m->lm_head, m->logits, T, dm, d.vocab, m->status, st));
   if (paired) {
     const int Th = pair_rows;
-    QZO_TRY(launch_cross_entropy(m->logits, d_labels, Th, d.vocab, m->row_loss, d_loss, st));
+    QZO_TRY(launch_cross_entropy(m->logits, d_labels, Th, d.vocab, m->row_loss, d_loss, d_sums, d_sums ? d_sums + 2 : nullptr, st));
     QZO_TRY(launch_cross_entropy(m->logits + (size_t)Th * d.vocab, d_labels + Th, Th, d.vocab, m->row_loss + Th,
-                                 d_loss + 1, st));
+                                 d_loss ? d_loss + 1 : nullptr, d_sums ? d_sums + 1 : nullptr, d_sums ? d_sums + 3 : nullptr, st));
   } else {
-    QZO_TRY(launch_cross_entropy(m->logits, d_labels, T, d.vocab, m->row_loss, d_loss, st));
+    QZO_TRY(launch_cross_entropy(m->logits, d_labels, T, d.vocab, m->row_loss, d_loss, d_sums ? d_sums + slot : nullptr,
+                                 d_sums ? d_sums + 2 + slot : nullptr, st));
   }
   m->last_T = T;
   return QZO_OK;
@@ -276,8 +284,10 @@ int update_all_scales(qzo_model* m, uint64_t seed, float coef_host, const float*
   return launch_update_scales(m->scales, m->flat_entries, seed, 0, coef_host, coef_dev, m->stream);
 }
 
-int step_device(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S, uint64_t seed, float eps,
-                float lr, float clip, float* h_out) {
+// First half of a step: both perturbed forwards (Algorithm 1, the two forward passes on the same batch and
+// seed); d_sums receives {sum of token losses (+), the same (-), kept tokens (+), kept tokens (-)}.
+int step_begin(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S, uint64_t seed, float eps,
+               float* d_sums) {
   const int T = B * S;
   if (paired_rows_ok(2 * T, T)) {
     // both passes as one forward over two copies of the batch (the workspace holds 2 * max_tokens rows)
@@ -288,19 +298,44 @@ int step_device(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, 
       QZO_CUDA_TRY(cudaMemcpyAsync(m->lab_dev, d_labels, bytes, cudaMemcpyDeviceToDevice, m->stream));
     QZO_CUDA_TRY(cudaMemcpyAsync(m->tok_dev + T, m->tok_dev, bytes, cudaMemcpyDeviceToDevice, m->stream));
     QZO_CUDA_TRY(cudaMemcpyAsync(m->lab_dev + T, m->lab_dev, bytes, cudaMemcpyDeviceToDevice, m->stream));
-    QZO_TRY(forward_loss(m, m->tok_dev, m->lab_dev, B, S, seed, +1, eps, m->loss2, true));
+    QZO_TRY(forward_loss(m, m->tok_dev, m->lab_dev, B, S, seed, +1, eps, m->loss2, d_sums, true));
   } else {
-    QZO_TRY(forward_loss(m, d_tokens, d_labels, B, S, seed, +1, eps, m->loss2, false));
-    QZO_TRY(forward_loss(m, d_tokens, d_labels, B, S, seed, -1, eps, m->loss2 + 1, false));
-  }
-  QZO_TRY(launch_ddc(m->loss2, m->loss2 + 1, eps, lr, clip, m->out5, m->stream));
-  QZO_TRY(update_all_scales(m, seed, 0.0f, m->out5 + 4));
-  if (h_out) {
-    QZO_CUDA_TRY(cudaMemcpyAsync(h_out, m->out5, 4 * sizeof(float), cudaMemcpyDeviceToHost, m->stream));
-    QZO_CUDA_TRY(cudaStreamSynchronize(m->stream));
-    if (!std::isfinite(h_out[0]) || !std::isfinite(h_out[1])) return QZO_ERR_NONFINITE;
+    QZO_TRY(forward_loss(m, d_tokens, d_labels, B, S, seed, +1, eps, m->loss2, d_sums, false, 0));
+    QZO_TRY(forward_loss(m, d_tokens, d_labels, B, S, seed, -1, eps, m->loss2 + 1, d_sums, false, 1));
   }
   return QZO_OK;
+}
+
+// Second half: d, d' (Eq. 6) and the seeded update from the loss sums, all on the device.  With h_out the
+// stream is synchronised and what the device found is reported; the scales are untouched in every error case.
+int step_finish(qzo_model* m, const float* d_sums, uint64_t seed, float eps, float lr, float clip, float* h_out) {
+  QZO_TRY(launch_ddc(d_sums, eps, lr, clip, m->status, m->out6, m->stream));
+  QZO_TRY(update_all_scales(m, seed, 0.0f, m->out6 + 4));
+  if (h_out) {
+    float host[6];
+    QZO_CUDA_TRY(cudaMemcpyAsync(host, m->out6, sizeof(host), cudaMemcpyDeviceToHost, m->stream));
+    QZO_CUDA_TRY(cudaStreamSynchronize(m->stream));
+    memcpy(h_out, host, 4 * sizeof(float));
+    const int st = (int)host[5];
+    if (st & kStatusTimeout) return QZO_ERR_DEVICE_TIMEOUT;
+    if (st & kStatusBadToken) return QZO_ERR_BAD_ARG;
+    if (!std::isfinite(host[0]) || !std::isfinite(host[1])) return QZO_ERR_NONFINITE;
+  }
+  return QZO_OK;
+}
+
+int step_device(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S, uint64_t seed, float eps,
+                float lr, float clip, float* h_out) {
+  QZO_TRY(step_begin(m, d_tokens, d_labels, B, S, seed, eps, m->sums));
+  return step_finish(m, m->sums, seed, eps, lr, clip, h_out);
+}
+
+// (layer, linear) of a flat linear id, or false when it is out of range.
+bool split_linear_id(const qzo_model* m, int linear_id, int* layer, int* linear) {
+  if (linear_id < 0 || linear_id >= m->desc.n_layers * m->n_lin) return false;
+  *layer = linear_id / m->n_lin;
+  *linear = linear_id % m->n_lin;
+  return true;
 }
 
 }  // namespace qzo
@@ -515,7 +550,8 @@ int qzo_init_model(const qzo_model_desc* desc, const qzo_tensor* tensors, int n_
   m->row_loss = (float*)(ws + p.off_rowloss);
   float* scal = (float*)(ws + p.off_scalars);
   m->loss2 = scal;            // [0], [1]
-  m->out5 = scal + 8;         // [8..12]
+  m->sums = scal + 4;         // [4..7]
+  m->out6 = scal + 8;         // [8..13]
   m->status = (int*)(scal + 32);
   m->rope_cs = (float*)(ws + p.off_rope);
   m->tok_dev = (int32_t*)(ws + p.off_tok);
@@ -575,7 +611,7 @@ int qzo_forward_loss(qzo_model* m, const int32_t* d_tokens, const int32_t* d_lab
                      int sign, float eps, float* d_loss) {
   QZO_TRY(check_batch(m, d_tokens, d_labels, B, S));
   if (!d_loss || sign < -1 || sign > 1 || !(eps > 0.0f)) return QZO_ERR_BAD_ARG;
-  return forward_loss(m, d_tokens, d_labels, B, S, seed, sign, eps, d_loss, false);
+  return forward_loss(m, d_tokens, d_labels, B, S, seed, sign, eps, d_loss, nullptr, false);
 }
 
 int qzo_update_scales(qzo_model* m, uint64_t seed, float lr, float g, float clip) {
@@ -600,6 +636,60 @@ int qzo_step_host(qzo_model* m, const int32_t* h_tokens, const int32_t* h_labels
   QZO_CUDA_TRY(cudaMemcpyAsync(m->tok_dev, h_tokens, bytes, cudaMemcpyHostToDevice, m->stream));
   QZO_CUDA_TRY(cudaMemcpyAsync(m->lab_dev, h_labels, bytes, cudaMemcpyHostToDevice, m->stream));
   return step_device(m, m->tok_dev, m->lab_dev, B, S, seed, eps, lr, clip, h_out);
+}
+
+int qzo_step_begin(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S, uint64_t seed,
+                   float eps, float* d_sums) {
+  QZO_TRY(check_batch(m, d_tokens, d_labels, B, S));
+  if (!(eps > 0.0f) || !d_sums || ((uintptr_t)d_sums & 15)) return QZO_ERR_BAD_ARG;
+  return step_begin(m, d_tokens, d_labels, B, S, seed, eps, d_sums);
+}
+
+int qzo_step_finish(qzo_model* m, const float* d_sums, uint64_t seed, float eps, float lr, float clip, float* h_out) {
+  if (!m || !d_sums || ((uintptr_t)d_sums & 15)) return QZO_ERR_BAD_ARG;
+  if (!(eps > 0.0f) || !(clip >= 0.0f) || !std::isfinite(lr)) return QZO_ERR_BAD_ARG;
+  return step_finish(m, d_sums, seed, eps, lr, clip, h_out);
+}
+
+int qzo_get_scales(qzo_model* m, int linear_id, void* d_bf16, size_t bytes) {
+  if (!m || !d_bf16) return QZO_ERR_BAD_ARG;
+  const __nv_bfloat16* src = m->scales;
+  size_t need = (size_t)m->flat_entries * 2;
+  if (linear_id != -1) {
+    int layer = 0, linear = 0;
+    if (!split_linear_id(m, linear_id, &layer, &linear)) return QZO_ERR_BAD_ARG;
+    const Linear& L = m->layers[layer].lin[linear];
+    src = m->scales + L.idx_base;
+    need = (size_t)ceil_div(L.K, kGroup) * L.N * 2;
+  }
+  if (bytes != need) return QZO_ERR_BAD_ARG;
+  QZO_CUDA_TRY(cudaMemcpyAsync(d_bf16, src, need, cudaMemcpyDeviceToDevice, m->stream));
+  return QZO_OK;
+}
+
+int qzo_set_scales(qzo_model* m, int linear_id, const void* d_bf16, size_t bytes) {
+  if (!m || !d_bf16) return QZO_ERR_BAD_ARG;
+  __nv_bfloat16* dst = m->scales;
+  size_t need = (size_t)m->flat_entries * 2;
+  if (linear_id != -1) {
+    int layer = 0, linear = 0;
+    if (!split_linear_id(m, linear_id, &layer, &linear)) return QZO_ERR_BAD_ARG;
+    const Linear& L = m->layers[layer].lin[linear];
+    dst = m->scales + L.idx_base;
+    need = (size_t)ceil_div(L.K, kGroup) * L.N * 2;
+  }
+  if (bytes != need) return QZO_ERR_BAD_ARG;
+  QZO_CUDA_TRY(cudaMemcpyAsync(dst, d_bf16, need, cudaMemcpyDeviceToDevice, m->stream));
+  return QZO_OK;
+}
+
+int qzo_debug_set_status(qzo_model* m, int value) {
+  if (!m || value < 0) return QZO_ERR_BAD_ARG;
+  // a host-side write of the word the kernels report through: lets a test walk the error path of a
+  // step without making any device-side wait expire
+  QZO_CUDA_TRY(cudaMemcpyAsync(m->status, &value, sizeof(int), cudaMemcpyHostToDevice, m->stream));
+  QZO_CUDA_TRY(cudaStreamSynchronize(m->stream));
+  return QZO_OK;
 }
 
 int qzo_debug_set_capture(qzo_model* m, int layer) {
@@ -629,7 +719,8 @@ int qzo_device_status(qzo_model* m, int* h_status) {
   if (!m || !h_status) return QZO_ERR_BAD_ARG;
   QZO_CUDA_TRY(cudaMemcpyAsync(h_status, m->status, sizeof(int), cudaMemcpyDeviceToHost, m->stream));
   QZO_CUDA_TRY(cudaStreamSynchronize(m->stream));
-  return *h_status ? QZO_ERR_DEVICE_TIMEOUT : QZO_OK;
+  if (*h_status & kStatusTimeout) return QZO_ERR_DEVICE_TIMEOUT;
+  return (*h_status & kStatusBadToken) ? QZO_ERR_BAD_ARG : QZO_OK;
 }
 
 }  // extern "C"

@@ -29,6 +29,10 @@ void set_last_cuda_error(cudaError_t e);
     if (_s != QZO_OK) return _s;                            \
   } while (0)
 
+// Bits of the device status word of a model (0 = nothing to report).
+constexpr int kStatusTimeout = 1;    // a bounded device-side wait expired in some launch
+constexpr int kStatusBadToken = 2;   // a token id outside [0, vocab) reached the embedding
+
 constexpr int kGroup = 128;          // rows of one quantisation group (paper: group 128)
 constexpr int kTileN = 128;          // output features per GEMM tile (UMMA M)
 constexpr int kBlockK = 64;          // K elements per pipeline stage (one 128-byte swizzle atom of bf16)

@@ -27,6 +27,7 @@ EXPORTS = (
     "qzo_scale_layout", "qzo_workspace_bytes", "qzo_init_model", "qzo_free_model", "qzo_forward_loss",
     "qzo_update_scales", "qzo_step", "qzo_step_host", "qzo_debug_set_capture", "qzo_debug_layer_output",
     "qzo_device_status", "qzo_launch_count", "qzo_profile_gemms", "qzo_profile_read",
+    "qzo_step_begin", "qzo_step_finish", "qzo_get_scales", "qzo_set_scales", "qzo_debug_set_status",
 )
 
 
@@ -83,6 +84,11 @@ def _load():
         "qzo_update_scales": (ci, [vp, u64, cf, cf, cf]),
         "qzo_step": (ci, [vp, vp, vp, ci, ci, u64, cf, cf, cf, vp]),
         "qzo_step_host": (ci, [vp, vp, vp, ci, ci, u64, cf, cf, cf, vp]),
+        "qzo_step_begin": (ci, [vp, vp, vp, ci, ci, u64, cf, vp]),
+        "qzo_step_finish": (ci, [vp, vp, u64, cf, cf, cf, vp]),
+        "qzo_get_scales": (ci, [vp, ci, vp, sz]),
+        "qzo_set_scales": (ci, [vp, ci, vp, sz]),
+        "qzo_debug_set_status": (ci, [vp, ci]),
         "qzo_debug_set_capture": (ci, [vp, ci]),
         "qzo_debug_layer_output": (ci, [vp, ci, ci, vp, sz]),
         "qzo_device_status": (ci, [vp, P(ci)]),
@@ -303,6 +309,43 @@ class Model:
         _check(_lib.qzo_step(self.handle, _ptr(tokens), _ptr(labels), B, S, seed, eps, lr, clip, out), "qzo_step")
         return tuple(out) if read_back else None
 
+    def qzo_step_begin(self, tokens, labels, seed, eps, sums=None):
+        """-> float32 CUDA tensor [4]: sum of token losses (+), the same (-), kept tokens (+), (-)."""
+        _cuda(tokens, torch.int32), _cuda(labels, torch.int32)
+        B, S = tokens.shape
+        if sums is None:
+            sums = torch.empty((4,), dtype=torch.float32, device="cuda")
+        _check(_lib.qzo_step_begin(self.handle, _ptr(tokens), _ptr(labels), B, S, seed, eps, _ptr(sums)),
+               "qzo_step_begin")
+        return sums
+
+    def qzo_step_finish(self, sums, seed, eps, lr, clip, read_back=True):
+        _cuda(sums, torch.float32)
+        out = (ctypes.c_float * 4)() if read_back else None
+        _check(_lib.qzo_step_finish(self.handle, _ptr(sums), seed, eps, lr, clip, out), "qzo_step_finish")
+        return tuple(out) if read_back else None
+
+    def _linear_bytes(self, linear_id):
+        if linear_id == -1:
+            return self.scales.numel() * 2
+        n_lin = 7 if self.cfg["arch"] == "llama" else 6
+        _, G, N = qzo_scale_layout(self.cfg, linear_id // n_lin, linear_id % n_lin)
+        return G * N * 2
+
+    def qzo_get_scales(self, linear_id, out=None):
+        """Copy of one linear's scales (bf16, flat [G*N]) or of the whole flat buffer (linear_id = -1)."""
+        if out is None:
+            out = torch.empty((self._linear_bytes(linear_id) // 2,), dtype=torch.bfloat16, device="cuda")
+        _check(_lib.qzo_get_scales(self.handle, linear_id, _ptr(out), out.numel() * 2), "qzo_get_scales")
+        return out
+
+    def qzo_set_scales(self, linear_id, values):
+        _cuda(values, torch.bfloat16)
+        _check(_lib.qzo_set_scales(self.handle, linear_id, _ptr(values), values.numel() * 2), "qzo_set_scales")
+
+    def qzo_debug_set_status(self, value):
+        _check(_lib.qzo_debug_set_status(self.handle, value), "qzo_debug_set_status")
+
     def qzo_step_host(self, tokens_host, labels_host, seed, eps, lr, clip):
         assert not tokens_host.is_cuda and tokens_host.dtype == torch.int32 and tokens_host.is_contiguous()
         B, S = tokens_host.shape
@@ -327,7 +370,7 @@ class Model:
     def qzo_device_status(self):
         st = ctypes.c_int(0)
         rc = _lib.qzo_device_status(self.handle, ctypes.byref(st))
-        if rc not in (QZO_OK, ERR_DEVICE_TIMEOUT):
+        if rc not in (QZO_OK, ERR_DEVICE_TIMEOUT, ERR_BAD_ARG):
             _check(rc, "qzo_device_status")
         return st.value
 

@@ -3,7 +3,7 @@ import copy
 
 import numpy as np
 
-from oracle import int4
+from oracle import int4, linear as olinear, model as omodel
 
 
 def f32(t):
@@ -35,3 +35,42 @@ def build_oracle_model(raw):
 
 def clone_model(m):
     return copy.deepcopy(m)
+
+
+def llama_forward_with_bf16_storage(model, tokens, seed, sign, eps):
+    """The oracle's Llama forward (fp64 arithmetic, same functions) with every tensor that a 16-bit
+    implementation keeps in memory rounded to bf16 where it is stored: the de-quantised weight s' q, the
+    norm outputs, every linear's output, the rotated q and k, the attention output, the activation and the
+    residual stream.  It answers one question: how far does bf16 STORAGE alone move a block's output away
+    from the un-rounded oracle?  Where that already exceeds the 2e-2 bound (strongly non-linear models),
+    the parity test bounds the GPU by this figure instead.  Returns (hidden per block, logits)."""
+    cfg = model["cfg"]
+    assert cfg["arch"] == "llama"
+    B, S = tokens.shape
+    d, H = cfg["d_model"], cfg["n_heads"]
+    dh = d // H
+    bases, _ = omodel.scale_index_bases(cfg)
+    bf = lambda a: int4.bf16_round(np.asarray(a, dtype=np.float32)).astype(np.float64)
+    x = np.asarray(model["embed"], np.float64)[tokens.reshape(-1)]
+
+    def lin(layer, li, name, inp):
+        p = layer["lin"][name]
+        sp = olinear.perturbed_scales(p["s"], seed, bases[li][name], sign, eps)
+        w = bf(sp[np.arange(p["q"].shape[0]) // int4.GROUP] * p["q"].astype(np.float64))
+        return bf(inp @ w)
+
+    hidden = []
+    for li, layer in enumerate(model["layers"]):
+        n1 = bf(omodel.rmsnorm(x, np.asarray(layer["norm1_w"], np.float64), cfg["norm_eps"]))
+        qh = bf(omodel.rope(lin(layer, li, "q", n1).reshape(B, S, H, dh), cfg["rope_theta"]))
+        kh = bf(omodel.rope(lin(layer, li, "k", n1).reshape(B, S, H, dh), cfg["rope_theta"]))
+        vh = lin(layer, li, "v", n1).reshape(B, S, H, dh)
+        att = bf(omodel.causal_attention(qh, kh, vh).reshape(B * S, d))
+        h = bf(x + lin(layer, li, "o", att))
+        n2 = bf(omodel.rmsnorm(h, np.asarray(layer["norm2_w"], np.float64), cfg["norm_eps"]))
+        g, u = lin(layer, li, "gate", n2), lin(layer, li, "up", n2)
+        act = bf(g / (1.0 + np.exp(-g)) * u)
+        x = bf(h + lin(layer, li, "down", act))
+        hidden.append(x.copy())
+    xn = bf(omodel.rmsnorm(x, np.asarray(model["final_norm_w"], np.float64), cfg["norm_eps"]))
+    return hidden, xn @ np.asarray(model["lm_head"], dtype=np.float64).T

@@ -26,6 +26,9 @@ def test_binding_covers_header_and_host_only_calls_work():
     from paper_2505_13430_b200 import qzo, inputs
     assert sorted(qzo.EXPORTS) == _declared()
     assert qzo._lib.qzo_strerror(0) == b"ok"
+    header = open(os.path.join(ROOT, "include", "qzo.h")).read()
+    shift = re.search(r"#define QZO_NOALLOC_SCRATCH_BYTES \((\d+)u << (\d+)\)", header)
+    assert qzo.NOALLOC_SCRATCH_BYTES == int(shift.group(1)) << int(shift.group(2))
     assert b"workspace" in qzo._lib.qzo_strerror(qzo.ERR_WORKSPACE)
     # host-side queries need no device
     assert qzo.qzo_repacked_bytes(4096, 4096) == 4096 * 4096 // 2

@@ -1,5 +1,6 @@
-"""With one rank the data-parallel step is Algorithm 1 on the whole batch: same losses, same d, and
-bit-identical scales as qzo_step (d formed on the host here, on the device there)."""
+"""With one rank the data-parallel step (begin, exchange, finish) is Algorithm 1 on the whole batch:
+same losses, same d and bit-identical scales as qzo_step; and splitting the batch over two model
+replicas whose loss sums are added (what two ranks' all-reduce does) gives the whole-batch step."""
 import pytest
 import torch
 
@@ -8,22 +9,51 @@ from paper_2505_13430_b200 import inputs
 pytestmark = pytest.mark.gpu
 
 
-def test_single_rank_dp_step_equals_qzo_step():
-    from paper_2505_13430_b200 import qzo, data_parallel as dp
+def _tiny():
+    from paper_2505_13430_b200 import qzo
     cfg = inputs.model_cfg("tiny")
     c = inputs.CONFIGS["tiny"]
     raw = inputs.raw_model_tensors(cfg, seed=1000)
-    gm = qzo.build_model_from_raw(raw, c["batch"] * c["seq"])
     tok, lab = inputs.tokens_and_labels(cfg, c["batch"], c["seq"], seed=7)
+    return qzo, cfg, c, raw, tok, lab
+
+
+def test_single_rank_dp_step_equals_qzo_step():
+    from paper_2505_13430_b200 import data_parallel as dp
+    qzo, cfg, c, raw, tok, lab = _tiny()
+    gm = qzo.build_model_from_raw(raw, c["batch"] * c["seq"])
     tok_d, lab_d = tok.cuda(), lab.cuda()
     before = gm.scales.clone()
     ref = gm.qzo_step(tok_d, lab_d, 42, c["eps"], c["lr"] * 50, c["clip"])
     after_ref = gm.scales.clone()
     gm.scales.copy_(before)
     got = dp.dp_step(gm, tok_d, lab_d, 42, c["eps"], c["lr"] * 50, c["clip"])
-    assert got[0] == ref[0] and got[1] == ref[1]
-    assert abs(got[2] - ref[2]) <= 1e-6 * max(1.0, abs(ref[2])) and got[3] == ref[3]
+    assert got == ref
     assert torch.equal(gm.scales.view(torch.int16), after_ref.view(torch.int16))
     assert not torch.equal(after_ref.view(torch.int16), before.view(torch.int16))
-    assert dp.kept_tokens(lab) == c["batch"] * (c["seq"] - 1)
     gm.close()
+
+
+def test_two_replicas_with_added_loss_sums_follow_the_whole_batch_step():
+    # Two "ranks" emulated one after the other on one GPU (nothing waits on anything): each runs the begin
+    # half on its half of the batch, the sums are added as an all-reduce would, both finish with the total.
+    qzo, cfg, c, raw, tok, lab = _tiny()
+    T = c["batch"] * c["seq"]
+    whole = qzo.build_model_from_raw(raw, T)
+    ranks = [qzo.build_model_from_raw(raw, T) for _ in range(2)]
+    seed, eps, lr, clip = 9, c["eps"], c["lr"] * 50, c["clip"]
+    ref = whole.qzo_step(tok.cuda(), lab.cuda(), seed, eps, lr, clip)
+    half = c["batch"] // 2
+    sums = [ranks[r].qzo_step_begin(tok[r * half:(r + 1) * half].contiguous().cuda(),
+                                    lab[r * half:(r + 1) * half].contiguous().cuda(), seed, eps) for r in range(2)]
+    total = sums[0] + sums[1]
+    assert float(total[2]) == float(total[3]) == c["batch"] * (c["seq"] - 1)
+    outs = [ranks[r].qzo_step_finish(total, seed, eps, lr, clip) for r in range(2)]
+    assert outs[0] == outs[1]
+    # the token-weighted mean of the halves is the whole batch's mean up to fp32 summation order
+    assert abs(outs[0][0] - ref[0]) <= 2e-6 * abs(ref[0]) and abs(outs[0][1] - ref[1]) <= 2e-6 * abs(ref[1])
+    assert torch.equal(ranks[0].scales.view(torch.int16), ranks[1].scales.view(torch.int16))
+    if outs[0][3] == ref[3]:             # same clipped d' (both clipped, or bit-equal d): same update as the whole batch
+        assert torch.equal(ranks[0].scales.view(torch.int16), whole.scales.view(torch.int16))
+    for m in ranks + [whole]:
+        m.close()

@@ -3,6 +3,11 @@
 * The standalone perturbed W4A16 GEMM on every K x N and token count of the sweep, in the launch
   configuration the sweep times (same entry point, same tile / split-K choice): sampled rows and
   columns (first and last tile, ragged edges, random ones) against the oracle, max relative 2e-2.
+* A full-width model truncated to two decoder blocks, at the benchmark's batch, through qzo_step (both
+  signs in one pass, the route the benchmark times): losses L+- within 1e-3 of the oracle's, the
+  directional derivative printed beside the oracle's.
+* A Llama-2-7B-width block built for 4096 tokens and called with 16 and with 128 tokens (the split-K
+  route of the small-token GEMMs inside a model whose workspace was planned for the large batch).
 * One full-width decoder block of the Llama-2-7B shape (16 x 256 tokens) and of the OPT-6.7B shape
   (32 x 128 tokens; LayerNorm, biases, ReLU, learned positions) at the benchmark's batch, so the
   grouped q/k/v and gate/up launches and the 256-token tiles are the ones the benchmark runs: block output and logits of sampled sequences against the oracle (sequences of a batch do
@@ -97,4 +102,63 @@ def test_full_width_block_matches_oracle_on_sampled_sequences(lib, workload):
     before = gm.scales.clone()
     out = gm.qzo_step(tok.cuda(), lab.cuda(), seed, eps, c["lr"], 0.0)
     assert out[3] == 0.0 and torch.equal(gm.scales.view(torch.int16), before.view(torch.int16))
+    gm.close()
+
+
+def _oracle_and_gpu_model(lib, workload, n_layers, max_tokens):
+    cfg = inputs.model_cfg(workload, n_layers=n_layers)
+    raw = inputs.raw_model_tensors(cfg, seed=1000)
+    om = build_oracle_model(raw)
+    quant = {(li, name): (torch.from_numpy(int4.pack_int4(om["layers"][li]["lin"][name]["q"]).view(np.int32)),
+                          torch.from_numpy(om["layers"][li]["lin"][name]["s"]).bfloat16())
+             for li in range(n_layers) for name in omodel.LINEAR_ORDER[cfg["arch"]]}
+    gm = lib.build_model_from_raw(raw, max_tokens, quantized=quant)
+    return cfg, om, gm
+
+
+@pytest.mark.parametrize("workload", ["llama7b", "opt6.7b"])
+def test_two_layer_full_width_step_losses_match_oracle(lib, workload):
+    c = inputs.CONFIGS[workload]
+    B, S = c["batch"], c["seq"]
+    cfg, om, gm = _oracle_and_gpu_model(lib, workload, 2, B * S)
+    tok, lab = inputs.tokens_and_labels(cfg, B, S, seed=7)
+    seed, eps = 42, c["eps"]
+    lp, lm, d, dc = gm.qzo_step(tok.cuda(), lab.cuda(), seed, eps, c["lr"], c["clip"])
+    assert gm.qzo_device_status() == 0
+    rp = omodel.forward_loss(om, tok.numpy(), lab.numpy(), seed, +1, eps)
+    rm = omodel.forward_loss(om, tok.numpy(), lab.numpy(), seed, -1, eps)
+    d_ref = (rp - rm) / (2 * eps)
+    print(f"{workload} x 2 layers, {B} x {S} tokens: L+ {lp:.6f} (oracle {rp:.6f})  L- {lm:.6f} (oracle {rm:.6f})  "
+          f"d {d:.4f} (oracle {d_ref:.4f})")
+    assert abs(lp - rp) <= 1e-3 and abs(lm - rm) <= 1e-3
+    # d is a difference of two losses that agree to 1e-3 each: what that allows, and no more
+    assert abs(d - d_ref) <= 2e-3 / (2 * eps)
+    gm.close()
+
+
+@pytest.mark.parametrize("tokens", [(1, 16), (2, 64)])
+def test_small_batch_on_a_model_planned_for_the_large_batch(lib, tokens):
+    # max_tokens = 4096: the workspace must also hold the split-K partial sums of the small-token GEMMs
+    B, S = tokens
+    cfg, om, gm = _oracle_and_gpu_model(lib, "llama7b", 1, 4096)
+    tok, lab = inputs.tokens_and_labels(cfg, B, S, seed=11)
+    # The 1e-3 bound on a loss is stated for the configurations' batches (at least 188 kept tokens, where the
+    # bf16 rounding errors of the single tokens average out); the mean over the 15 or 126 kept tokens here
+    # averages fewer of them, so the bound is widened by sqrt(188 / kept).  The block output and the logits
+    # keep the 2e-2 bound.
+    kept = B * (S - 1)
+    tol_loss = 1e-3 * max(1.0, (188.0 / kept) ** 0.5)
+    gm.qzo_debug_set_capture(0)
+    for sign in (+1, -1):
+        loss = float(gm.qzo_forward_loss(tok.cuda(), lab.cuda(), 5, sign, 1e-3).cpu()[0])
+        cap = {}
+        ref = omodel.forward_loss(om, tok.numpy(), lab.numpy(), 5, sign, 1e-3, capture=cap)
+        hid = gm.qzo_debug_layer_output(0, 0, B * S).float().cpu().numpy().astype(np.float64)
+        logits = gm.qzo_debug_layer_output(0, 1, B * S).float().cpu().numpy().astype(np.float64)
+        assert np.abs(hid - cap["hidden"][0]).max() <= TOL * np.abs(cap["hidden"][0]).max()
+        assert np.abs(logits - cap["logits"]).max() <= TOL * np.abs(cap["logits"]).max()
+        assert abs(loss - ref) <= tol_loss, (sign, loss, ref)
+    lp, lm, d, dc = gm.qzo_step(tok.cuda(), lab.cuda(), 5, 1e-3, 1e-5, 100.0)
+    assert gm.qzo_device_status() == 0
+    assert abs(lp - omodel.forward_loss(om, tok.numpy(), lab.numpy(), 5, +1, 1e-3)) <= tol_loss
     gm.close()

@@ -7,7 +7,7 @@ import torch
 
 from oracle import model as omodel, qzo as oqzo
 from paper_2505_13430_b200 import inputs
-from tests.helpers import build_oracle_model, clone_model
+from tests.helpers import build_oracle_model, clone_model, llama_forward_with_bf16_storage
 
 pytestmark = pytest.mark.gpu
 
@@ -44,7 +44,8 @@ def _bf16_ulp_diff(a, b):
     return (key(a) - key(b)).abs()
 
 
-@pytest.mark.parametrize("name,gain", [("tiny", 1.0), ("tiny", 3.0), ("tiny_opt", 1.0), ("tiny_opt", 3.0), ("tiny_dh128", 3.0)])
+@pytest.mark.parametrize("name,gain", [("tiny", 1.0), ("tiny", 3.0), ("tiny", 6.0), ("tiny_opt", 1.0), ("tiny_opt", 3.0),
+                                       ("tiny_opt", 4.0), ("tiny_dh128", 3.0)])
 def test_forward_and_step_match_oracle(lib, name, gain):
     cfg, c, om, gm, tok, lab = _setup(lib, name, gain)
     T = c["batch"] * c["seq"]
@@ -59,13 +60,23 @@ def test_forward_and_step_match_oracle(lib, name, gain):
     for sign in (+1, -1, 0):
         cap = {}
         ref_loss = omodel.forward_loss(om, tok.numpy(), lab.numpy(), seed, sign, eps, capture=cap)
+        # Bound on a block's output: 2e-2, except where storing the intermediates in bf16 ALONE (fp64
+        # arithmetic otherwise) already moves the oracle further than that; this happens only for the
+        # strongly non-linear gain-6 model (2.2e-2 / 2.6e-2), and the bound is then that figure + 25 %.
+        tol_h, tol_l = [2e-2] * cfg["n_layers"], 2e-2
+        if gain >= 6.0:
+            emu_h, emu_l = llama_forward_with_bf16_storage(om, tok.numpy(), seed, sign, eps)
+            inherent = [np.abs(emu_h[li] - cap["hidden"][li]).max() / np.abs(cap["hidden"][li]).max()
+                        for li in range(cfg["n_layers"])]
+            tol_h = [max(2e-2, 1.25 * v) for v in inherent]
+            tol_l = max(2e-2, 1.25 * np.abs(emu_l - cap["logits"]).max() / np.abs(cap["logits"]).max())
         for li in range(cfg["n_layers"]):
             gm.qzo_debug_set_capture(li)
             loss = float(gm.qzo_forward_loss(tok_d, lab_d, seed, sign, eps).cpu()[0])
             hid = gm.qzo_debug_layer_output(li, 0, T)
-            assert _relerr(hid, cap["hidden"][li]) <= 2e-2, (sign, li)
+            assert _relerr(hid, cap["hidden"][li]) <= tol_h[li], (sign, li, _relerr(hid, cap["hidden"][li]))
         logits = gm.qzo_debug_layer_output(0, 1, T)
-        assert _relerr(logits, cap["logits"]) <= 2e-2
+        assert _relerr(logits, cap["logits"]) <= tol_l
         assert abs(loss - ref_loss) <= 1e-3, (sign, loss, ref_loss)
         losses[sign] = (loss, ref_loss)
     assert gm.qzo_device_status() == 0
@@ -105,6 +116,18 @@ def test_forward_and_step_match_oracle(lib, name, gain):
     gm.scales.copy_(before)
     gm.qzo_update_scales(seed, lr, d, clip)
     assert torch.equal(gm.scales.view(torch.int16), after_dev.view(torch.int16))
+    # a threshold below |d|: the clip branch of Eq. 6 on the device against the oracle's, and the update it drives
+    if abs(d) > 1e-3:
+        c_small = float(np.float32(abs(d) / 2))
+        gm.scales.copy_(before)
+        out = gm.qzo_step(tok_d, lab_d, seed, eps, lr * 50, c_small)
+        assert out[2] == d and out[3] == np.float32(oqzo.ddc_clip(d, c_small)) and abs(out[3]) == c_small
+        om3 = clone_model(om)
+        oqzo.update_model_scales(om3, seed, lr * 50, oqzo.ddc_clip(d, c_small))
+        for li in range(cfg["n_layers"]):
+            for i, nm in enumerate(order):
+                ref = torch.from_numpy(om3["layers"][li]["lin"][nm]["s"]).bfloat16()
+                assert int(_bf16_ulp_diff(gm.scales_of(li, i).cpu(), ref).max()) <= 1
     # C = 0: d' = 0 and the scales stay bit-identical
     gm.scales.copy_(before)
     out = gm.qzo_step(tok_d, lab_d, seed, eps, lr, 0.0)
@@ -185,4 +208,69 @@ def test_step_in_one_pass_equals_two_separate_passes(lib, name):
         ref_m = omodel.forward_loss(om, t.numpy(), l.numpy(), seed, -1, eps)
         assert abs(out[0] - ref_p) <= 1e-3 and abs(out[1] - ref_m) <= 1e-3, rows
     assert gm.qzo_device_status() == 0
+    gm.close()
+
+
+def test_get_and_set_scales_round_trip(lib):
+    # The trainable state goes out and comes back through the C ABI: set -> step -> get equals the flat
+    # buffer's slice bit for bit, sizes are checked, and a saved state resumes a run exactly.
+    cfg, c, om, gm, tok, lab = _setup(lib, "tiny")
+    n_lin = 7
+    lid = 1 * n_lin + 6                                      # layer 1, "down": K = 688 (short last group)
+    base, G, N = lib.qzo_scale_layout(cfg, 1, 6)
+    new = (torch.rand((G * N,), device="cuda") * 0.01 + 0.005).bfloat16()
+    gm.qzo_set_scales(lid, new)
+    assert torch.equal(gm.scales[base:base + G * N].view(torch.int16), new.view(torch.int16))
+    saved = gm.qzo_get_scales(-1)
+    assert torch.equal(saved.view(torch.int16), gm.scales.view(torch.int16))
+    tok_d, lab_d = tok.cuda(), lab.cuda()
+    out1 = gm.qzo_step(tok_d, lab_d, 5, c["eps"], c["lr"] * 50, c["clip"])
+    got = gm.qzo_get_scales(lid)
+    assert torch.equal(got.view(torch.int16), gm.scales[base:base + G * N].view(torch.int16))
+    assert not torch.equal(got.view(torch.int16), new.view(torch.int16))
+    after1 = gm.qzo_get_scales(-1)
+    gm.qzo_set_scales(-1, saved)                             # resume from the saved state: same step, same result
+    out2 = gm.qzo_step(tok_d, lab_d, 5, c["eps"], c["lr"] * 50, c["clip"])
+    assert out2 == out1 and torch.equal(gm.qzo_get_scales(-1).view(torch.int16), after1.view(torch.int16))
+    for bad_id, t in ((n_lin * cfg["n_layers"], new), (-2, new), (lid, new[:-8].contiguous()), (0, new)):
+        with pytest.raises(lib.QzoError) as e:
+            gm.qzo_set_scales(bad_id, t)
+        assert e.value.status == lib.ERR_BAD_ARG
+    with pytest.raises(lib.QzoError) as e:
+        gm.qzo_get_scales(lid, out=torch.empty((G * N + 8,), dtype=torch.bfloat16, device="cuda"))
+    assert e.value.status == lib.ERR_BAD_ARG
+    gm.close()
+
+
+def test_reported_device_failure_leaves_the_scales_untouched(lib):
+    # The failure is made on the host: the status word that a kernel sets when one of its bounded waits
+    # expires is written with a host-side copy.  The step must then return the error and change nothing.
+    cfg, c, om, gm, tok, lab = _setup(lib, "tiny")
+    tok_d, lab_d = tok.cuda(), lab.cuda()
+    before = gm.scales.clone()
+    gm.qzo_debug_set_status(1)
+    with pytest.raises(lib.QzoError) as e:
+        gm.qzo_step(tok_d, lab_d, 42, c["eps"], c["lr"] * 50, c["clip"])
+    assert e.value.status == lib.ERR_DEVICE_TIMEOUT
+    assert torch.equal(gm.scales.view(torch.int16), before.view(torch.int16))
+    gm.qzo_step(tok_d, lab_d, 42, c["eps"], c["lr"] * 50, c["clip"], read_back=False)     # also without a read-back
+    torch.cuda.synchronize()
+    assert torch.equal(gm.scales.view(torch.int16), before.view(torch.int16))
+    assert gm.qzo_device_status() == 1
+    gm.qzo_debug_set_status(0)
+    gm.qzo_step(tok_d, lab_d, 42, c["eps"], c["lr"] * 50, c["clip"])
+    assert not torch.equal(gm.scales.view(torch.int16), before.view(torch.int16))
+    gm.close()
+
+
+def test_token_id_out_of_range_is_reported(lib):
+    cfg, c, om, gm, tok, lab = _setup(lib, "tiny")
+    bad = tok.clone()
+    bad[1, 3] = cfg["vocab"]                                 # one past the last valid id
+    before = gm.scales.clone()
+    with pytest.raises(lib.QzoError) as e:
+        gm.qzo_step(bad.cuda(), lab.cuda(), 42, c["eps"], c["lr"] * 50, c["clip"])
+    assert e.value.status == lib.ERR_BAD_ARG
+    assert torch.equal(gm.scales.view(torch.int16), before.view(torch.int16))
+    assert gm.qzo_device_status() == 2
     gm.close()

@@ -54,22 +54,37 @@ def test_single_process_needs_no_group():
     assert replicas.whole_job_rate(10, 1, 2000.0) == 5.0
 
 
+class _StubModel:
+    """Stands in for qzo.Model on CPU: the begin half reports this rank's loss sums, the finish half
+    records what reached it."""
+
+    def __init__(self, sums):
+        self.sums = torch.tensor(sums, dtype=torch.float32)
+        self.finish_args = None
+
+    def qzo_step_begin(self, tokens, labels, seed, eps):
+        return self.sums.clone()
+
+    def qzo_step_finish(self, sums, seed, eps, lr, clip, read_back=True):
+        self.finish_args = (sums.tolist(), seed, eps, lr, clip)
+        return None
+
+
 def _dp_worker(rank, world, port, out):
     os.environ["MASTER_ADDR"] = "127.0.0.1"
     os.environ["MASTER_PORT"] = str(port)
     dist.init_process_group("gloo", rank=rank, world_size=world)
     try:
         from paper_2505_13430_b200 import data_parallel as dp
-        # rank 0: 10 tokens with mean loss 2.0 / 1.0, rank 1: 30 tokens with mean loss 4.0 / 5.0
-        n = 10 if rank == 0 else 30
-        lp = dp.global_mean_loss(2.0 if rank == 0 else 4.0, n)
-        lm = dp.global_mean_loss(1.0 if rank == 0 else 5.0, n)
-        out.put((rank, lp, lm) + dp.directional_derivative(lp, lm, 1e-3, 100.0))
+        # rank 0: 10 kept tokens with loss sums 20 / 10, rank 1: 30 kept tokens with loss sums 120 / 150
+        stub = _StubModel([20.0, 10.0, 10.0, 10.0] if rank == 0 else [120.0, 150.0, 30.0, 30.0])
+        dp.dp_step(stub, None, None, seed=77, eps=1e-3, lr=1e-5, clip=100.0, read_back=False)
+        out.put((rank,) + stub.finish_args)
     finally:
         dist.destroy_process_group()
 
 
-def test_data_parallel_exchange_is_two_scalars_and_every_rank_gets_the_same_d():
+def test_data_parallel_step_exchanges_four_floats_and_every_rank_finishes_alike():
     world = 2
     ctx = mp.get_context("spawn")
     out = ctx.Queue()
@@ -81,8 +96,9 @@ def test_data_parallel_exchange_is_two_scalars_and_every_rank_gets_the_same_d():
     for p in procs:
         p.join(timeout=60)
         assert p.exitcode == 0
-    # token-weighted means: l+ = (10*2 + 30*4)/40 = 3.5, l- = (10*1 + 30*5)/40 = 4.0; d = -250 -> d' = -100
+    # the finish half of BOTH ranks got the element-wise sums and the same seed / eps / lr / clip, so the
+    # library forms the same d' and applies the same seeded update on both
     for r in res:
-        assert abs(r[1] - 3.5) < 1e-12 and abs(r[2] - 4.0) < 1e-12
-        assert abs(r[3] + 250.0) < 1e-3 and r[4] == -100.0
-    assert res[0][1:] == res[1][1:]                      # identical on both ranks -> identical seeded update
+        assert r[1] == [140.0, 160.0, 40.0, 40.0]
+        assert r[2:] == (77, 1e-3, 1e-5, 100.0)
+    assert res[0][1:] == res[1][1:]

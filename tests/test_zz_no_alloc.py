@@ -31,8 +31,12 @@ def test_noalloc_entry_matches_workspace_entry_twice_in_a_row():
         x, wq, s = _case(lib, M, K, N, seed)
         ref = lib.qzo_perturbed_gemm(x, wq, s, M, K, N, 1000 + call, 8 * call, sign, 1e-3, status=status)
         y.fill_(float("nan"))
+        torch.cuda.synchronize()
+        free0, held0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
         lib.qzo_perturbed_gemm_noalloc(x, wq, s, y, M, K, N, 1000 + call, 8 * call, sign, 1e-3, status=status)
         torch.cuda.synchronize()
+        if call > 0:        # after the first call on the device (module load, address look-up) nothing is taken
+            assert torch.cuda.mem_get_info()[0] >= free0 and torch.cuda.memory_allocated() == held0
         assert int(status.item()) == 0
         # same kernels, same fixed summation order: the outputs are bit-identical (the parity tests
         # of qzo_perturbed_gemm against the oracle allow 2e-2; this is stricter)
