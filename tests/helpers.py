@@ -74,3 +74,11 @@ def llama_forward_with_bf16_storage(model, tokens, seed, sign, eps):
         hidden.append(x.copy())
     xn = bf(omodel.rmsnorm(x, np.asarray(model["final_norm_w"], np.float64), cfg["norm_eps"]))
     return hidden, xn @ np.asarray(model["lm_head"], dtype=np.float64).T
+
+
+def loss_tolerance(kept_tokens):
+    """Bound on |L_gpu - L_oracle| for a mean over `kept_tokens` positions.  The 1e-3 of the method's
+    configurations is stated for their batches (the smallest keeps 188 positions), where the bf16 rounding
+    errors of the single tokens' losses (a few 1e-3 each, independent from token to token) average out; a
+    mean over fewer positions averages fewer of them, so the bound widens by sqrt(188 / kept)."""
+    return 1e-3 * max(1.0, (188.0 / max(int(kept_tokens), 1)) ** 0.5)

@@ -71,7 +71,10 @@ CASES = [
     (300, 1024, 384),      # two token tiles, ragged M
     (1, 512, 256),         # single token
     (130, 384, 1000),      # N tail 104, 3 groups
-    (16, 4096, 4096),      # split-K path
+    (8, 1024, 384),        # streaming kernel, one token tile of 8
+    (5, 688, 688),         # streaming kernel: K tail, N tail, ragged M
+    (9, 11008, 192),       # streaming kernel: 86 groups, CTAs share every output block
+    (16, 4096, 4096),      # streaming kernel at a sweep size
     (128, 4096, 512),      # split-K with M = 128
     (257, 2048, 1024),     # 256-token tile + 1
 ]
