@@ -60,6 +60,42 @@ def scale_index_bases(cfg):
     return bases, run
 
 
+def dense_tensor_names(cfg):
+    """The un-quantised tensors that joint SPSA also perturbs and updates, in index order:
+    (key, layer or None).  Embedding and lm_head matrices, then every norm gain (and norm bias, OPT)."""
+    opt = cfg["arch"] == "opt"
+    names = [("embed", None), ("lm_head", None)]
+    for li in range(cfg["n_layers"]):
+        names.append(("norm1_w", li))
+        if opt:
+            names.append(("norm1_b", li))
+        names.append(("norm2_w", li))
+        if opt:
+            names.append(("norm2_b", li))
+    names.append(("final_norm_w", None))
+    if opt:
+        names.append(("final_norm_b", None))
+    return names
+
+
+def dense_tensor(model, key, layer):
+    return model[key] if layer is None else model["layers"][layer][key]
+
+
+def dense_index_bases(cfg):
+    """Logical indices of the un-quantised tensors under joint SPSA: they follow the scales in the same
+    z(seed, index) stream (so one seed still regenerates every direction), each base rounded up to a
+    multiple of 8.  Returns ({(key, layer): base}, total)."""
+    _, run = scale_index_bases(cfg)
+    d, V = cfg["d_model"], cfg["vocab"]
+    out = {}
+    for key, layer in dense_tensor_names(cfg):
+        run = (run + 7) // 8 * 8
+        out[(key, layer)] = run
+        run += V * d if key in ("embed", "lm_head") else d
+    return out, run
+
+
 def num_trainable_scales(cfg):
     return sum(num_groups(K) * N for _, K, N in linear_shapes(cfg)) * cfg["n_layers"]
 
@@ -108,34 +144,51 @@ def cross_entropy(logits, labels):
     return float(np.sum((lse - picked)[keep]) / max(int(keep.sum()), 1))
 
 
-def forward_loss(model, tokens, labels, seed, sign, eps, capture=None):
+def forward_loss(model, tokens, labels, seed, sign, eps, capture=None, perturb_scales=True,
+                 perturb_dense=False):
     """L(Delta' (.) theta_bar; B) with Delta' = Delta + sign*eps*z(seed).
+
+    perturb_dense: joint mode (Sec. 3.2.1, closing remark; Sec. 4.1): the un-quantised tensors
+    of dense_tensor_names are perturbed as well, theta' = theta + sign*eps*z (plain SPSA,
+    Def. 3.1), with z from the same seed at the indices of dense_index_bases.
+    perturb_scales=False leaves the scales alone (used to pin the dense part by itself).
 
     capture: optional dict filled with 'hidden' (list, output of every block,
     [T][d]) and 'logits' ([T][V]) for per-layer parity checks.
     """
+    from . import philox
     cfg = model["cfg"]
     tokens = np.asarray(tokens)
     B, S = tokens.shape
     d, H = cfg["d_model"], cfg["n_heads"]
     dh = d // H
     bases, _ = scale_index_bases(cfg)
-    x = np.asarray(model["embed"], dtype=np.float64)[tokens.reshape(-1)]
+    dbases, _ = dense_index_bases(cfg)
+    scale_sign = sign if perturb_scales else 0
+
+    def dense(key, layer=None):
+        """theta or theta + sign*eps*z of one un-quantised tensor, fp64."""
+        t = np.asarray(dense_tensor(model, key, layer), dtype=np.float64)
+        if not perturb_dense or sign == 0:
+            return t
+        z = philox.normal_range(seed, dbases[(key, layer)], t.size).astype(np.float64).reshape(t.shape)
+        return t + float(sign) * float(eps) * z          # Def. 3.1 (same as qzo.spsa_perturbed)
+
+    x = dense("embed")[tokens.reshape(-1)]
     if cfg["arch"] == "opt":
         pos = np.asarray(model["pos_embed"], dtype=np.float64)[:S]
         x = (x.reshape(B, S, d) + pos[None]).reshape(B * S, d)
 
     def lin(layer, li, name, inp):
         p = layer["lin"][name]
-        return perturbed_linear(inp, p["q"], p["s"], seed, bases[li][name], sign, eps,
+        return perturbed_linear(inp, p["q"], p["s"], seed, bases[li][name], scale_sign, eps,
                                 p.get("bias"))
 
     for li, layer in enumerate(model["layers"]):
         if cfg["arch"] == "llama":
-            n1 = rmsnorm(x, np.asarray(layer["norm1_w"], np.float64), cfg["norm_eps"])
+            n1 = rmsnorm(x, dense("norm1_w", li), cfg["norm_eps"])
         else:
-            n1 = layernorm(x, np.asarray(layer["norm1_w"], np.float64),
-                           np.asarray(layer["norm1_b"], np.float64), cfg["norm_eps"])
+            n1 = layernorm(x, dense("norm1_w", li), dense("norm1_b", li), cfg["norm_eps"])
         qh = lin(layer, li, "q", n1).reshape(B, S, H, dh)
         kh = lin(layer, li, "k", n1).reshape(B, S, H, dh)
         vh = lin(layer, li, "v", n1).reshape(B, S, H, dh)
@@ -144,24 +197,22 @@ def forward_loss(model, tokens, labels, seed, sign, eps, capture=None):
         att = causal_attention(qh, kh, vh).reshape(B * S, d)
         h = x + lin(layer, li, "o", att)
         if cfg["arch"] == "llama":
-            n2 = rmsnorm(h, np.asarray(layer["norm2_w"], np.float64), cfg["norm_eps"])
+            n2 = rmsnorm(h, dense("norm2_w", li), cfg["norm_eps"])
             g = lin(layer, li, "gate", n2)
             u = lin(layer, li, "up", n2)
             act = g / (1.0 + np.exp(-g)) * u
             x = h + lin(layer, li, "down", act)
         else:
-            n2 = layernorm(h, np.asarray(layer["norm2_w"], np.float64),
-                           np.asarray(layer["norm2_b"], np.float64), cfg["norm_eps"])
+            n2 = layernorm(h, dense("norm2_w", li), dense("norm2_b", li), cfg["norm_eps"])
             act = np.maximum(lin(layer, li, "fc1", n2), 0.0)
             x = h + lin(layer, li, "fc2", act)
         if capture is not None:
             capture.setdefault("hidden", []).append(x.copy())
     if cfg["arch"] == "llama":
-        xn = rmsnorm(x, np.asarray(model["final_norm_w"], np.float64), cfg["norm_eps"])
+        xn = rmsnorm(x, dense("final_norm_w"), cfg["norm_eps"])
     else:
-        xn = layernorm(x, np.asarray(model["final_norm_w"], np.float64),
-                       np.asarray(model["final_norm_b"], np.float64), cfg["norm_eps"])
-    logits = xn @ np.asarray(model["lm_head"], dtype=np.float64).T
+        xn = layernorm(x, dense("final_norm_w"), dense("final_norm_b"), cfg["norm_eps"])
+    logits = xn @ dense("lm_head").T
     if capture is not None:
         capture["logits"] = logits
     return cross_entropy(logits, labels)
