@@ -102,7 +102,7 @@ def test_dense_directional_derivative_matches_reverse_mode_gradients():
     assert abs(want) > 1.0
     assert errs[1] <= 5e-4 and 10.0 < errs[0] / errs[1] < 40.0
     # joint = scales part + dense part to first order (one z stream, disjoint index ranges)
-    eps = 1e-3
+    eps = 1e-4
     def dd(**kw):
         return qzo.directional_derivative(omodel.forward_loss(m, tok.numpy(), lab.numpy(), seed, +1, eps, **kw),
                                           omodel.forward_loss(m, tok.numpy(), lab.numpy(), seed, -1, eps, **kw), eps)
