@@ -227,6 +227,20 @@ int qzo_step_begin(qzo_model* m, const int32_t* d_tokens, const int32_t* d_label
 int qzo_step_finish(qzo_model* m, const float* d_sums, uint64_t seed, float eps, float lr, float clip,
                     float* h_out);
 
+/* Joint mode (Sec. 3.2.1, closing remark: Q-SPSA on the scales combined with SPSA on the un-quantised
+ * parts; Sec. 4.1: "the un-quantized parts are jointly fine-tuned using the regular SPSA and ZO-SGD").
+ * After qzo_enable_joint_spsa every perturbed forward (sign +1 / -1) also perturbs the embedding matrix, the
+ * lm_head matrix and every norm gain (and norm bias, OPT) as theta + sign eps z (Def. 3.1), and every step
+ * also updates them in place, theta <- theta - lr_dense d' z (Def. 3.2; no clamp, that belongs to the
+ * scales), with the same clipped d' as the scales.  z comes from the same (seed, index) stream at indices
+ * that follow the scales': each base rounded up to a multiple of 8, in the order embed, lm_head, then per
+ * layer norm1 gain (bias), norm2 gain (bias), then the final norm.  Position embeddings and the biases of
+ * the linears stay fixed.  The caller's "embed", "lm_head" and norm tensors must be writable.
+ * d_workspace: qzo_joint_workspace_bytes (perturbed copies of the vectors and of the lm_head for both
+ * signs), 256-aligned, must outlive the handle; NULL switches the mode off.  Synchronises the stream. */
+int qzo_joint_workspace_bytes(const qzo_model_desc* desc, size_t* bytes);
+int qzo_enable_joint_spsa(qzo_model* m, void* d_workspace, size_t workspace_bytes, float lr_dense);
+
 /* Same step with HOST token / label buffers (int32 [B][S]); copies them in, runs the step and
  * reads {l+, l-, d, d'} back.  Synchronises. */
 int qzo_step_host(qzo_model* m, const int32_t* h_tokens, const int32_t* h_labels, int B, int S,

@@ -28,4 +28,13 @@ int launch_repack(const uint32_t* d_packed, int K, int N, void* d_out, cudaStrea
 int launch_unpack_kernel_layout(const void* d_wq, int K, int N, int8_t* d_q, cudaStream_t st);
 int launch_update_scales(__nv_bfloat16* d_s, int64_t count, uint64_t seed, uint64_t index_base,
                          float coef_host, const float* coef_dev, cudaStream_t st);
+// joint mode: plain SPSA on the un-quantised tensors
+int launch_perturb_dense_bf16(const __nv_bfloat16* src, __nv_bfloat16* dst, int64_t count, uint64_t seed,
+                              uint64_t index_base, float sign_eps, cudaStream_t st);
+int launch_perturb_vectors(const float* const* src_table, const unsigned long long* base_table, int n_vec, int d,
+                           uint64_t seed, float eps, float* plus, float* minus, cudaStream_t st);
+int launch_update_dense_bf16(__nv_bfloat16* th, int64_t count, uint64_t seed, uint64_t index_base, const float* coef_dev,
+                             cudaStream_t st);
+int launch_update_vectors(float* const* table, const unsigned long long* base_table, int n_vec, int d, uint64_t seed,
+                          const float* coef_dev, cudaStream_t st);
 }  // namespace qzo

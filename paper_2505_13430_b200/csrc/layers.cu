@@ -2,6 +2,7 @@
 // RoPE, causal attention, MLP activations, fused cross entropy, and the scalar kernel that
 // forms d and d' (Algorithm 1; Eq. 6).  All arithmetic is fp32 on bf16 storage.
 #include "qzo_common.cuh"
+#include "philox.cuh"
 #include "launch.cuh"
 #include "layers.cuh"
 
@@ -45,23 +46,38 @@ __device__ __forceinline__ float block_max(float v, float* red) {
 // A token id outside [0, vocab) sets bit 1 of the status word (the step then reports a bad argument and
 // leaves the scales alone); the row is still written, from the nearest valid id, so nothing is read
 // out of bounds.
+// Joint mode (pert.sign_eps != 0): the embedding row is perturbed as E + sign eps z (Def. 3.1) with z at
+// index pert.base + tok * d + j; rows from pert.pair_rows on (the second copy of a paired step) take -eps.
+struct EmbedPerturb { unsigned long long seed, base; float sign_eps; int pair_rows; };
+
 __global__ void embedding_kernel(const int32_t* __restrict__ tokens, const __nv_bfloat16* __restrict__ embed,
                                  const __nv_bfloat16* __restrict__ pos, int S, int d, int vocab,
-                                 __nv_bfloat16* __restrict__ x, int* __restrict__ status) {
+                                 __nv_bfloat16* __restrict__ x, int* __restrict__ status, EmbedPerturb pert) {
   const int t = blockIdx.x;
   int tok = tokens[t];
   if ((tok < 0 || tok >= vocab) && threadIdx.x == 0 && status != nullptr) atomicOr(status, kStatusBadToken);
   tok = min(max(tok, 0), vocab - 1);
-  const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(embed + (size_t)tok * d);
-  const __nv_bfloat162* pp = pos ? reinterpret_cast<const __nv_bfloat162*>(pos + (size_t)(t % S) * d) : nullptr;
-  __nv_bfloat162* o = reinterpret_cast<__nv_bfloat162*>(x + (size_t)t * d);
-  for (int i = threadIdx.x; i < d / 2; i += blockDim.x) {
-    float2 v = __bfloat1622float2(e[i]);
-    if (pp) {
-      const float2 q = __bfloat1622float2(pp[i]);
-      v.x += q.x; v.y += q.y;
+  const uint2* e = reinterpret_cast<const uint2*>(embed + (size_t)tok * d);
+  const uint2* pp = pos ? reinterpret_cast<const uint2*>(pos + (size_t)(t % S) * d) : nullptr;
+  uint2* o = reinterpret_cast<uint2*>(x + (size_t)t * d);
+  const float se = (pert.pair_rows > 0 && t >= pert.pair_rows) ? -pert.sign_eps : pert.sign_eps;
+  for (int i = threadIdx.x; i < d / 4; i += blockDim.x) {       // four elements = one counter block (d % 8 == 0)
+    uint2 raw = e[i];
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
+    float2 a = __bfloat1622float2(h[0]), b = __bfloat1622float2(h[1]);
+    if (se != 0.0f) {
+      float z[4];
+      normals_of_block(pert.seed, (pert.base + (unsigned long long)tok * (unsigned long long)d) / 4 + (unsigned long long)i, z);
+      a.x = fmaf(se, z[0], a.x); a.y = fmaf(se, z[1], a.y); b.x = fmaf(se, z[2], b.x); b.y = fmaf(se, z[3], b.y);
     }
-    o[i] = __floats2bfloat162_rn(v.x, v.y);
+    if (pp) {
+      const uint2 praw = pp[i];
+      const __nv_bfloat162* ph = reinterpret_cast<const __nv_bfloat162*>(&praw);
+      const float2 c = __bfloat1622float2(ph[0]), e2 = __bfloat1622float2(ph[1]);
+      a.x += c.x; a.y += c.y; b.x += e2.x; b.y += e2.y;
+    }
+    __nv_bfloat162 out[2] = {__floats2bfloat162_rn(a.x, a.y), __floats2bfloat162_rn(b.x, b.y)};
+    o[i] = *reinterpret_cast<const uint2*>(out);
   }
 }
 
@@ -77,7 +93,10 @@ constexpr int kNormVecs = 4;
 template <bool LAYERNORM>
 __global__ void __launch_bounds__(kNormThreads)
 add_norm_kernel(__nv_bfloat16* __restrict__ x, const __nv_bfloat16* delta, const float* __restrict__ w,
-                const float* __restrict__ b, float eps, int d, __nv_bfloat16* y) {
+                const float* __restrict__ b, const float* __restrict__ w2, const float* __restrict__ b2, int pair_rows,
+                float eps, int d, __nv_bfloat16* y) {
+  // rows from pair_rows on (second copy of a paired step in joint mode) use the second gain / bias set
+  if (pair_rows > 0 && (int)blockIdx.x >= pair_rows) { w = w2; b = b2; }
   __shared__ float red[32];
   const int nvec = d >> 3;
   uint4* xrow = reinterpret_cast<uint4*>(x + (size_t)blockIdx.x * d);
@@ -455,9 +474,9 @@ __global__ void ce_mean_kernel(const float* __restrict__ row_loss, const int32_t
 // sums = {sum of token losses with +eps z, the same with -eps z, kept tokens of each pass}:
 // l+- = sum / count; d = (l+ - l-) / (2 eps); d' = clip(d, -C, C) (Eq. 6); coef = lr * d', forced to 0
 // (no update) when a loss is not finite or the status word reports a failed launch or a bad token.
-// out = {l+, l-, d, d', coef, status word as a float}
-__global__ void ddc_kernel(const float* __restrict__ sums, float eps, float lr, float clip, const int* __restrict__ status,
-                           float* __restrict__ out) {
+// out = {l+, l-, d, d', coef, status word as a float, coef of the un-quantised tensors (joint mode)}
+__global__ void ddc_kernel(const float* __restrict__ sums, float eps, float lr, float lr_dense, float clip,
+                           const int* __restrict__ status, float* __restrict__ out) {
   const float a = sums[0] / fmaxf(sums[2], 1.0f), b = sums[1] / fmaxf(sums[3], 1.0f);
   const float d = (a - b) / (2.0f * eps);
   const float dc = fminf(fmaxf(d, -clip), clip);
@@ -466,25 +485,29 @@ __global__ void ddc_kernel(const float* __restrict__ sums, float eps, float lr, 
   out[0] = a; out[1] = b; out[2] = d; out[3] = dc;
   out[4] = good ? __fmul_rn(lr, dc) : 0.0f;
   out[5] = (float)st;
+  out[6] = good ? __fmul_rn(lr_dense, dc) : 0.0f;    // joint mode: step of the un-quantised tensors
 }
 
 }  // namespace
 
 int launch_embedding(const int32_t* tokens, const __nv_bfloat16* embed, const __nv_bfloat16* pos, int T, int S, int d,
-                     int vocab, __nv_bfloat16* x, int* status, cudaStream_t st) {
-  QZO_LAUNCH(embedding_kernel, dim3(T), dim3(128), 0, st, tokens, embed, pos, S, d, vocab, x, status);
+                     int vocab, __nv_bfloat16* x, int* status, uint64_t seed, uint64_t index_base, float sign_eps,
+                     int pair_rows, cudaStream_t st) {
+  if ((d % 8) || (index_base % 4)) return QZO_ERR_BAD_ARG;
+  const EmbedPerturb pert{seed, index_base, sign_eps, pair_rows};
+  QZO_LAUNCH(embedding_kernel, dim3(T), dim3(128), 0, st, tokens, embed, pos, S, d, vocab, x, status, pert);
   return QZO_OK;
 }
-int launch_add_rmsnorm(__nv_bfloat16* x, const __nv_bfloat16* delta, const float* w, float eps, int T, int d,
-                       __nv_bfloat16* y, cudaStream_t st) {
+int launch_add_rmsnorm(__nv_bfloat16* x, const __nv_bfloat16* delta, const float* w, const float* w2, int pair_rows,
+                       float eps, int T, int d, __nv_bfloat16* y, cudaStream_t st) {
   if ((d % 8) || d > kNormVecs * kNormThreads * 8) return QZO_ERR_BAD_ARG;
-  QZO_LAUNCH(add_norm_kernel<false>, dim3(T), dim3(kNormThreads), 0, st, x, delta, w, nullptr, eps, d, y);
+  QZO_LAUNCH(add_norm_kernel<false>, dim3(T), dim3(kNormThreads), 0, st, x, delta, w, nullptr, w2, nullptr, pair_rows, eps, d, y);
   return QZO_OK;
 }
-int launch_add_layernorm(__nv_bfloat16* x, const __nv_bfloat16* delta, const float* w, const float* b, float eps,
-                         int T, int d, __nv_bfloat16* y, cudaStream_t st) {
+int launch_add_layernorm(__nv_bfloat16* x, const __nv_bfloat16* delta, const float* w, const float* b, const float* w2,
+                         const float* b2, int pair_rows, float eps, int T, int d, __nv_bfloat16* y, cudaStream_t st) {
   if ((d % 8) || d > kNormVecs * kNormThreads * 8) return QZO_ERR_BAD_ARG;
-  QZO_LAUNCH(add_norm_kernel<true>, dim3(T), dim3(kNormThreads), 0, st, x, delta, w, b, eps, d, y);
+  QZO_LAUNCH(add_norm_kernel<true>, dim3(T), dim3(kNormThreads), 0, st, x, delta, w, b, w2, b2, pair_rows, eps, d, y);
   return QZO_OK;
 }
 int launch_rope_table(float* cs, int max_seq, int dh, float theta, cudaStream_t st) {
@@ -537,8 +560,9 @@ int launch_cross_entropy(const float* logits, const int32_t* labels, int T, int 
   QZO_LAUNCH(ce_mean_kernel, dim3(1), dim3(1024), 0, st, row_loss, labels, T, V, loss, sum_out, count_out);
   return QZO_OK;
 }
-int launch_ddc(const float* sums4, float eps, float lr, float clip, const int* status, float* out6, cudaStream_t st) {
-  QZO_LAUNCH(ddc_kernel, dim3(1), dim3(1), 0, st, sums4, eps, lr, clip, status, out6);
+int launch_ddc(const float* sums4, float eps, float lr, float lr_dense, float clip, const int* status, float* out7,
+               cudaStream_t st) {
+  QZO_LAUNCH(ddc_kernel, dim3(1), dim3(1), 0, st, sums4, eps, lr, lr_dense, clip, status, out7);
   return QZO_OK;
 }
 

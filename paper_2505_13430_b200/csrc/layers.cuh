@@ -3,13 +3,16 @@
 #include "qzo_common.cuh"
 
 namespace qzo {
+// sign_eps != 0: rows are perturbed as E + sign_eps z(seed, index_base + tok d + j); rows from pair_rows on take -sign_eps
 int launch_embedding(const int32_t* tokens, const __nv_bfloat16* embed, const __nv_bfloat16* pos, int T, int S, int d,
-                     int vocab, __nv_bfloat16* x, int* status, cudaStream_t st);
-// x <- x + delta (skipped when delta is null), then y = norm(x); y may alias delta.
-int launch_add_rmsnorm(__nv_bfloat16* x, const __nv_bfloat16* delta, const float* w, float eps, int T, int d,
-                       __nv_bfloat16* y, cudaStream_t st);
-int launch_add_layernorm(__nv_bfloat16* x, const __nv_bfloat16* delta, const float* w, const float* b, float eps,
-                         int T, int d, __nv_bfloat16* y, cudaStream_t st);
+                     int vocab, __nv_bfloat16* x, int* status, uint64_t seed, uint64_t index_base, float sign_eps,
+                     int pair_rows, cudaStream_t st);
+// x <- x + delta (skipped when delta is null), then y = norm(x); y may alias delta.  pair_rows > 0: rows from
+// pair_rows on use the gains (and biases) w2 (b2).
+int launch_add_rmsnorm(__nv_bfloat16* x, const __nv_bfloat16* delta, const float* w, const float* w2, int pair_rows,
+                       float eps, int T, int d, __nv_bfloat16* y, cudaStream_t st);
+int launch_add_layernorm(__nv_bfloat16* x, const __nv_bfloat16* delta, const float* w, const float* b, const float* w2,
+                         const float* b2, int pair_rows, float eps, int T, int d, __nv_bfloat16* y, cudaStream_t st);
 int launch_rope_table(float* cs, int max_seq, int dh, float theta, cudaStream_t st);
 int launch_rope(__nv_bfloat16* q, __nv_bfloat16* k, int ldq, int ldk, const float* cs, int T, int S, int H, int dh,
                 cudaStream_t st);
@@ -20,8 +23,9 @@ int launch_relu(__nv_bfloat16* x, int64_t n, cudaStream_t st);
 // loss (mean), sum_out and count_out may each be null
 int launch_cross_entropy(const float* logits, const int32_t* labels, int T, int V, float* row_loss, float* loss,
                          float* sum_out, float* count_out, cudaStream_t st);
-// sums4 = {sum l+, sum l-, kept tokens (+), kept tokens (-)}; out6 = {l+, l-, d, d', lr d' or 0, status}
-int launch_ddc(const float* sums4, float eps, float lr, float clip, const int* status, float* out6, cudaStream_t st);
+// sums4 = {sum l+, sum l-, kept tokens (+), kept tokens (-)}; out7 = {l+, l-, d, d', lr d' or 0, status, lr_dense d' or 0}
+int launch_ddc(const float* sums4, float eps, float lr, float lr_dense, float clip, const int* status, float* out7,
+               cudaStream_t st);
 
 // gemm_w4a16.cu
 constexpr int kMaxSplitTokens = 128;   // launches with more tokens never split along K

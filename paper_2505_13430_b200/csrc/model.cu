@@ -110,13 +110,22 @@ struct qzo_model {
   // workspace regions
   __nv_bfloat16 *x = nullptr, *xn = nullptr, *qkv = nullptr, *att = nullptr, *mlp_a = nullptr, *mlp_b = nullptr,
                 *capture = nullptr;
-  float *logits = nullptr, *row_loss = nullptr, *loss2 = nullptr, *sums = nullptr, *out6 = nullptr, *rope_cs = nullptr;
+  float *logits = nullptr, *row_loss = nullptr, *loss2 = nullptr, *sums = nullptr, *out7 = nullptr, *rope_cs = nullptr;
   int32_t *tok_dev = nullptr, *lab_dev = nullptr;
   void* gemm_ws = nullptr;
   size_t gemm_ws_bytes = 0;
   int* status = nullptr;
   int capture_layer = -1;
   int last_T = 0;
+  // joint mode (plain SPSA on the un-quantised tensors), off unless qzo_enable_joint_spsa was called
+  bool joint = false;
+  float lr_dense = 0.0f;
+  int n_vec = 0;                              // norm gain / bias vectors, in the order of the index ranges
+  int64_t base_embed = 0, base_lm_head = 0;   // logical indices of the two matrices
+  const float* const* vec_table = nullptr;    // device: pointers to the vectors
+  const unsigned long long* vec_base = nullptr;   // device: their logical index bases
+  float *vec_plus = nullptr, *vec_minus = nullptr;   // perturbed copies [n_vec][d]
+  __nv_bfloat16 *lm_plus = nullptr, *lm_minus = nullptr;   // perturbed copies of the lm_head [V][d]
   // optional per-GEMM timing (CUDA events around every perturbed GEMM launch)
   bool profiling = false;
   std::vector<cudaEvent_t> events;
@@ -175,11 +184,27 @@ int plan_workspace(const qzo_model_desc& d, int max_tokens, WsPlan* p) {
 
 // x += delta (when delta is given), then out = norm(x): the residual add of a block's projection is
 // fused into the norm that follows it.
-static int add_norm(qzo_model* m, __nv_bfloat16* x, const __nv_bfloat16* delta, const float* w, const float* b, int T,
-                    __nv_bfloat16* out) {
+// vec: position of the gain among the joint mode's vectors (its bias, if any, follows it); sign and
+// pair_rows say which perturbed copy a row takes in joint mode (sign 0: the stored vectors).
+static int add_norm(qzo_model* m, __nv_bfloat16* x, const __nv_bfloat16* delta, const float* w, const float* b, int vec,
+                    int sign, int pair_rows, int T, __nv_bfloat16* out) {
+  const float *w2 = nullptr, *b2 = nullptr;
+  int pr = 0;
+  if (m->joint && sign != 0) {
+    const size_t d = m->desc.d_model;
+    const float* first = sign > 0 ? m->vec_plus : m->vec_minus;
+    const float* second = sign > 0 ? m->vec_minus : m->vec_plus;
+    w = first + (size_t)vec * d;
+    if (b) b = first + (size_t)(vec + 1) * d;
+    if (pair_rows > 0) {
+      pr = pair_rows;
+      w2 = second + (size_t)vec * d;
+      if (b) b2 = second + (size_t)(vec + 1) * d;
+    }
+  }
   if (m->desc.arch == QZO_ARCH_LLAMA)
-    return launch_add_rmsnorm(x, delta, w, m->desc.norm_eps, T, m->desc.d_model, out, m->stream);
-  return launch_add_layernorm(x, delta, w, b, m->desc.norm_eps, T, m->desc.d_model, out, m->stream);
+    return launch_add_rmsnorm(x, delta, w, w2, pr, m->desc.norm_eps, T, m->desc.d_model, out, m->stream);
+  return launch_add_layernorm(x, delta, w, b, w2, b2, pr, m->desc.norm_eps, T, m->desc.d_model, out, m->stream);
 }
 
 // Up to three block linears that read the same input, in one launch.
@@ -225,13 +250,17 @@ int forward_loss(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels,
   const int T = B * S;
   cudaStream_t st = m->stream;
   const bool llama = d.arch == QZO_ARCH_LLAMA;
-  QZO_TRY(launch_embedding(d_tokens, m->embed, llama ? nullptr : m->pos_embed, T, S, dm, d.vocab, m->x, m->status, st));
+  const bool jp = m->joint && sign != 0;            // joint mode: the un-quantised tensors are perturbed too
+  const int vpl = llama ? 2 : 4;                    // vectors per layer: norm1 gain (bias), norm2 gain (bias)
+  if (jp) QZO_TRY(launch_perturb_vectors(m->vec_table, m->vec_base, m->n_vec, dm, seed, eps, m->vec_plus, m->vec_minus, st));
+  QZO_TRY(launch_embedding(d_tokens, m->embed, llama ? nullptr : m->pos_embed, T, S, dm, d.vocab, m->x, m->status, seed,
+                           (uint64_t)m->base_embed, jp ? (float)sign * eps : 0.0f, jp ? pair_rows : 0, st));
   // The residual stream x is updated lazily: a projection writes its output to xn, and the norm that
   // follows adds it to x before normalising (x += xn; xn = norm(x)).
   const __nv_bfloat16* pending = nullptr;          // projection output not yet added to x
   for (int li = 0; li < d.n_layers; ++li) {
     const Layer& L = m->layers[li];
-    QZO_TRY(add_norm(m, m->x, pending, L.norm1_w, L.norm1_b, T, m->xn));
+    QZO_TRY(add_norm(m, m->x, pending, L.norm1_w, L.norm1_b, li * vpl, sign, pair_rows, T, m->xn));
     if (li > 0 && li - 1 == m->capture_layer)
       QZO_CUDA_TRY(cudaMemcpyAsync(m->capture, m->x, (size_t)T * dm * 2, cudaMemcpyDeviceToDevice, st));
     {
@@ -242,7 +271,7 @@ int forward_loss(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels,
     if (llama) QZO_TRY(launch_rope(m->qkv, m->qkv + dm, 3 * dm, 3 * dm, m->rope_cs, T, S, H, dh, st));
     QZO_TRY(launch_attention(m->qkv, m->qkv + dm, m->qkv + 2 * dm, 3 * dm, 3 * dm, 3 * dm, m->att, dm, B, S, H, dh, st));
     QZO_TRY(linear(m, L.lin[3], m->att, m->xn, dm, T, seed, sign, eps, pair_rows));
-    QZO_TRY(add_norm(m, m->x, m->xn, L.norm2_w, L.norm2_b, T, m->xn));
+    QZO_TRY(add_norm(m, m->x, m->xn, L.norm2_w, L.norm2_b, li * vpl + vpl / 2, sign, pair_rows, T, m->xn));
     if (llama) {
       const Linear* gu_l[2] = {&L.lin[4], &L.lin[5]};
       __nv_bfloat16* gu_o[2] = {m->mlp_a, m->mlp_b};
@@ -256,10 +285,26 @@ int forward_loss(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels,
     }
     pending = m->xn;
   }
-  QZO_TRY(add_norm(m, m->x, pending, m->final_norm_w, m->final_norm_b, T, m->xn));
+  QZO_TRY(add_norm(m, m->x, pending, m->final_norm_w, m->final_norm_b, d.n_layers * vpl, sign, pair_rows, T, m->xn));
   if (d.n_layers - 1 == m->capture_layer)
     QZO_CUDA_TRY(cudaMemcpyAsync(m->capture, m->x, (size_t)T * dm * 2, cudaMemcpyDeviceToDevice, st));
-  QZO_TRY(launch_bf16_gemm_f32out(m->xn, m->lm_head, m->logits, T, dm, d.vocab, m->status, st));
+  if (jp) {
+    // perturbed copies of the lm_head, rounded to its storage type; a paired pass needs both
+    const int64_t cnt = (int64_t)d.vocab * dm;
+    __nv_bfloat16* first = sign > 0 ? m->lm_plus : m->lm_minus;
+    QZO_TRY(launch_perturb_dense_bf16(m->lm_head, first, cnt, seed, (uint64_t)m->base_lm_head, (float)sign * eps, st));
+    if (paired) {
+      __nv_bfloat16* second = sign > 0 ? m->lm_minus : m->lm_plus;
+      QZO_TRY(launch_perturb_dense_bf16(m->lm_head, second, cnt, seed, (uint64_t)m->base_lm_head, -(float)sign * eps, st));
+      QZO_TRY(launch_bf16_gemm_f32out(m->xn, first, m->logits, pair_rows, dm, d.vocab, m->status, st));
+      QZO_TRY(launch_bf16_gemm_f32out(m->xn + (size_t)pair_rows * dm, second, m->logits + (size_t)pair_rows * d.vocab,
+                                      T - pair_rows, dm, d.vocab, m->status, st));
+    } else {
+      QZO_TRY(launch_bf16_gemm_f32out(m->xn, first, m->logits, T, dm, d.vocab, m->status, st));
+    }
+  } else {
+    QZO_TRY(launch_bf16_gemm_f32out(m->xn, m->lm_head, m->logits, T, dm, d.vocab, m->status, st));
+  }
   if (paired) {
     const int Th = pair_rows;
     QZO_TRY(launch_cross_entropy(m->logits, d_labels, Th, d.vocab, m->row_loss, d_loss, d_sums, d_sums ? d_sums + 2 : nullptr, st));
@@ -309,11 +354,20 @@ int step_begin(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, i
 // Second half: d, d' (Eq. 6) and the seeded update from the loss sums, all on the device.  With h_out the
 // stream is synchronised and what the device found is reported; the scales are untouched in every error case.
 int step_finish(qzo_model* m, const float* d_sums, uint64_t seed, float eps, float lr, float clip, float* h_out) {
-  QZO_TRY(launch_ddc(d_sums, eps, lr, clip, m->status, m->out6, m->stream));
-  QZO_TRY(update_all_scales(m, seed, 0.0f, m->out6 + 4));
+  QZO_TRY(launch_ddc(d_sums, eps, lr, m->joint ? m->lr_dense : 0.0f, clip, m->status, m->out7, m->stream));
+  QZO_TRY(update_all_scales(m, seed, 0.0f, m->out7 + 4));
+  if (m->joint) {
+    // ZO-SGD on the un-quantised tensors with the same clipped d' and the same z stream (Def. 3.2)
+    const int64_t cnt = (int64_t)m->desc.vocab * m->desc.d_model;
+    const float* coef = m->out7 + 6;
+    QZO_TRY(launch_update_dense_bf16(const_cast<__nv_bfloat16*>(m->embed), cnt, seed, (uint64_t)m->base_embed, coef, m->stream));
+    QZO_TRY(launch_update_dense_bf16(const_cast<__nv_bfloat16*>(m->lm_head), cnt, seed, (uint64_t)m->base_lm_head, coef, m->stream));
+    QZO_TRY(launch_update_vectors(const_cast<float* const*>(reinterpret_cast<const float* const*>(m->vec_table)), m->vec_base,
+                                  m->n_vec, m->desc.d_model, seed, coef, m->stream));
+  }
   if (h_out) {
     float host[6];
-    QZO_CUDA_TRY(cudaMemcpyAsync(host, m->out6, sizeof(host), cudaMemcpyDeviceToHost, m->stream));
+    QZO_CUDA_TRY(cudaMemcpyAsync(host, m->out7, sizeof(host), cudaMemcpyDeviceToHost, m->stream));
     QZO_CUDA_TRY(cudaStreamSynchronize(m->stream));
     memcpy(h_out, host, 4 * sizeof(float));
     const int st = (int)host[5];
@@ -551,7 +605,7 @@ int qzo_init_model(const qzo_model_desc* desc, const qzo_tensor* tensors, int n_
   float* scal = (float*)(ws + p.off_scalars);
   m->loss2 = scal;            // [0], [1]
   m->sums = scal + 4;         // [4..7]
-  m->out6 = scal + 8;         // [8..13]
+  m->out7 = scal + 8;         // [8..14]
   m->status = (int*)(scal + 32);
   m->rope_cs = (float*)(ws + p.off_rope);
   m->tok_dev = (int32_t*)(ws + p.off_tok);
@@ -649,6 +703,71 @@ int qzo_step_finish(qzo_model* m, const float* d_sums, uint64_t seed, float eps,
   if (!m || !d_sums || ((uintptr_t)d_sums & 15)) return QZO_ERR_BAD_ARG;
   if (!(eps > 0.0f) || !(clip >= 0.0f) || !std::isfinite(lr)) return QZO_ERR_BAD_ARG;
   return step_finish(m, d_sums, seed, eps, lr, clip, h_out);
+}
+
+static size_t joint_bytes(const qzo_model_desc& d, int* n_vec_out) {
+  const int n_vec = (2 * d.n_layers + 1) * (d.arch == QZO_ARCH_OPT ? 2 : 1);
+  if (n_vec_out) *n_vec_out = n_vec;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { off = (off + bytes + 255) / 256 * 256; };
+  take((size_t)n_vec * 8);                         // pointer table
+  take((size_t)n_vec * 8);                         // index bases
+  take((size_t)n_vec * d.d_model * 4);             // vectors, +eps
+  take((size_t)n_vec * d.d_model * 4);             // vectors, -eps
+  take((size_t)d.vocab * d.d_model * 2);           // lm_head, +eps
+  take((size_t)d.vocab * d.d_model * 2);           // lm_head, -eps
+  return off;
+}
+
+int qzo_joint_workspace_bytes(const qzo_model_desc* desc, size_t* bytes) {
+  QZO_TRY(validate_desc(desc));
+  if (!bytes) return QZO_ERR_BAD_ARG;
+  *bytes = joint_bytes(*desc, nullptr);
+  return QZO_OK;
+}
+
+int qzo_enable_joint_spsa(qzo_model* m, void* d_workspace, size_t workspace_bytes, float lr_dense) {
+  if (!m) return QZO_ERR_BAD_ARG;
+  if (!d_workspace) { m->joint = false; return QZO_OK; }
+  if (!std::isfinite(lr_dense)) return QZO_ERR_BAD_ARG;
+  if ((uintptr_t)d_workspace & 255) return QZO_ERR_WORKSPACE;
+  const qzo_model_desc& d = m->desc;
+  int n_vec = 0;
+  if (workspace_bytes < joint_bytes(d, &n_vec)) return QZO_ERR_WORKSPACE;
+  const bool opt = d.arch == QZO_ARCH_OPT;
+  // index ranges: after the scales, each base rounded up to a multiple of 8: embedding, lm_head, then the
+  // norm vectors layer by layer (gain, bias), the final norm last
+  int64_t run = m->flat_entries;
+  auto next_base = [&](int64_t count) { run = (run + 7) / 8 * 8; const int64_t b = run; run += count; return b; };
+  m->base_embed = next_base((int64_t)d.vocab * d.d_model);
+  m->base_lm_head = next_base((int64_t)d.vocab * d.d_model);
+  std::vector<const float*> ptrs;
+  std::vector<unsigned long long> bases;
+  auto add_vec = [&](const float* p) { ptrs.push_back(p); bases.push_back((unsigned long long)next_base(d.d_model)); };
+  for (int li = 0; li < d.n_layers; ++li) {
+    const Layer& L = m->layers[li];
+    add_vec(L.norm1_w); if (opt) add_vec(L.norm1_b);
+    add_vec(L.norm2_w); if (opt) add_vec(L.norm2_b);
+  }
+  add_vec(m->final_norm_w); if (opt) add_vec(m->final_norm_b);
+  uint8_t* ws = (uint8_t*)d_workspace;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { uint8_t* p = ws + off; off = (off + bytes + 255) / 256 * 256; return p; };
+  const float** tab = (const float**)take((size_t)n_vec * 8);
+  unsigned long long* bas = (unsigned long long*)take((size_t)n_vec * 8);
+  m->vec_plus = (float*)take((size_t)n_vec * d.d_model * 4);
+  m->vec_minus = (float*)take((size_t)n_vec * d.d_model * 4);
+  m->lm_plus = (__nv_bfloat16*)take((size_t)d.vocab * d.d_model * 2);
+  m->lm_minus = (__nv_bfloat16*)take((size_t)d.vocab * d.d_model * 2);
+  QZO_CUDA_TRY(cudaMemcpyAsync(tab, ptrs.data(), (size_t)n_vec * 8, cudaMemcpyHostToDevice, m->stream));
+  QZO_CUDA_TRY(cudaMemcpyAsync(bas, bases.data(), (size_t)n_vec * 8, cudaMemcpyHostToDevice, m->stream));
+  QZO_CUDA_TRY(cudaStreamSynchronize(m->stream));      // the host vectors go out of scope
+  m->vec_table = tab;
+  m->vec_base = bas;
+  m->n_vec = n_vec;
+  m->lr_dense = lr_dense;
+  m->joint = true;
+  return QZO_OK;
 }
 
 int qzo_get_scales(qzo_model* m, int linear_id, void* d_bf16, size_t bytes) {

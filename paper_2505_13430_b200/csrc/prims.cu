@@ -175,8 +175,113 @@ __global__ void update_scales_kernel(__nv_bfloat16* __restrict__ s, int64_t coun
 }
 
 // ---------------------------------------------------------------------------------------
+// Joint mode (Sec. 3.2.1, closing remark; Def. 3.1, Def. 3.2): the un-quantised tensors take plain
+// SPSA with z from the same (seed, index) stream, at indices that follow the scales'.
+// ---------------------------------------------------------------------------------------
+// dst_i = bf16(src_i + sign_eps z_i): perturbed copy of a bf16 matrix (the lm_head), four elements per
+// thread = one counter block; index_base is a multiple of 4, count a multiple of 4.
+__global__ void perturb_dense_bf16_kernel(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst,
+                                          int64_t count, uint64_t seed, uint64_t index_base, float sign_eps) {
+  const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t i0 = t * 4;
+  if (i0 >= count) return;
+  float z[4];
+  normals_of_block(seed, (index_base >> 2) + (uint64_t)t, z);
+  const uint2 raw = *reinterpret_cast<const uint2*>(src + i0);
+  __nv_bfloat16 v[4];
+  *reinterpret_cast<uint2*>(v) = raw;
+#pragma unroll
+  for (int l = 0; l < 4; ++l) v[l] = __float2bfloat16_rn(fmaf(sign_eps, z[l], __bfloat162float(v[l])));
+  *reinterpret_cast<uint2*>(dst + i0) = *reinterpret_cast<uint2*>(v);
+}
+
+// Perturbed copies of a set of fp32 vectors of length d (norm gains and biases): plus[v][j] = w + eps z,
+// minus[v][j] = w - eps z; src and base are device tables with one entry per vector.  grid = (ceil(d/4/256), n_vec).
+__global__ void perturb_vectors_kernel(const float* const* __restrict__ src, const unsigned long long* __restrict__ base,
+                                       int d, uint64_t seed, float eps, float* __restrict__ plus,
+                                       float* __restrict__ minus) {
+  const int v = blockIdx.y;
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  const int j0 = t * 4;
+  if (j0 >= d) return;
+  float z[4];
+  normals_of_block(seed, (base[v] >> 2) + (uint64_t)t, z);
+  const float4 w = *reinterpret_cast<const float4*>(src[v] + j0);
+  *reinterpret_cast<float4*>(plus + (size_t)v * d + j0) =
+      make_float4(fmaf(eps, z[0], w.x), fmaf(eps, z[1], w.y), fmaf(eps, z[2], w.z), fmaf(eps, z[3], w.w));
+  *reinterpret_cast<float4*>(minus + (size_t)v * d + j0) =
+      make_float4(fmaf(-eps, z[0], w.x), fmaf(-eps, z[1], w.y), fmaf(-eps, z[2], w.z), fmaf(-eps, z[3], w.w));
+}
+
+// ZO-SGD on an un-quantised bf16 matrix: theta_i <- bf16(theta_i - coef z_i); no clamp.
+__global__ void update_dense_bf16_kernel(__nv_bfloat16* __restrict__ th, int64_t count, uint64_t seed,
+                                         uint64_t index_base, const float* __restrict__ coef_dev) {
+  const float coef = *coef_dev;
+  if (coef == 0.0f) return;
+  const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t i0 = t * 4;
+  if (i0 >= count) return;
+  float z[4];
+  normals_of_block(seed, (index_base >> 2) + (uint64_t)t, z);
+  __nv_bfloat16 v[4];
+  *reinterpret_cast<uint2*>(v) = *reinterpret_cast<const uint2*>(th + i0);
+#pragma unroll
+  for (int l = 0; l < 4; ++l) v[l] = __float2bfloat16_rn(__fsub_rn(__bfloat162float(v[l]), __fmul_rn(coef, z[l])));
+  *reinterpret_cast<uint2*>(th + i0) = *reinterpret_cast<uint2*>(v);
+}
+
+// The same for a set of fp32 vectors (device tables as in perturb_vectors_kernel).
+__global__ void update_vectors_kernel(float* const* __restrict__ th, const unsigned long long* __restrict__ base, int d,
+                                      uint64_t seed, const float* __restrict__ coef_dev) {
+  const float coef = *coef_dev;
+  if (coef == 0.0f) return;
+  const int v = blockIdx.y;
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  const int j0 = t * 4;
+  if (j0 >= d) return;
+  float z[4];
+  normals_of_block(seed, (base[v] >> 2) + (uint64_t)t, z);
+  float4 w = *reinterpret_cast<const float4*>(th[v] + j0);
+  w.x = __fsub_rn(w.x, __fmul_rn(coef, z[0])); w.y = __fsub_rn(w.y, __fmul_rn(coef, z[1]));
+  w.z = __fsub_rn(w.z, __fmul_rn(coef, z[2])); w.w = __fsub_rn(w.w, __fmul_rn(coef, z[3]));
+  *reinterpret_cast<float4*>(th[v] + j0) = w;
+}
+
+// ---------------------------------------------------------------------------------------
 // Host launchers
 // ---------------------------------------------------------------------------------------
+int launch_perturb_dense_bf16(const __nv_bfloat16* src, __nv_bfloat16* dst, int64_t count, uint64_t seed,
+                              uint64_t index_base, float sign_eps, cudaStream_t st) {
+  if (count == 0) return QZO_OK;
+  if ((count % 4) || (index_base % 4)) return QZO_ERR_BAD_ARG;
+  QZO_LAUNCH(perturb_dense_bf16_kernel, dim3((unsigned)ceil_div64(count / 4, 256)), dim3(256), 0, st, src, dst, count, seed,
+             index_base, sign_eps);
+  return QZO_OK;
+}
+int launch_perturb_vectors(const float* const* src_table, const unsigned long long* base_table, int n_vec, int d,
+                           uint64_t seed, float eps, float* plus, float* minus, cudaStream_t st) {
+  if (n_vec == 0) return QZO_OK;
+  if (d % 4) return QZO_ERR_BAD_ARG;
+  QZO_LAUNCH(perturb_vectors_kernel, dim3(ceil_div(d / 4, 256), n_vec), dim3(256), 0, st, src_table, base_table, d, seed, eps,
+             plus, minus);
+  return QZO_OK;
+}
+int launch_update_dense_bf16(__nv_bfloat16* th, int64_t count, uint64_t seed, uint64_t index_base, const float* coef_dev,
+                             cudaStream_t st) {
+  if (count == 0) return QZO_OK;
+  if ((count % 4) || (index_base % 4)) return QZO_ERR_BAD_ARG;
+  QZO_LAUNCH(update_dense_bf16_kernel, dim3((unsigned)ceil_div64(count / 4, 256)), dim3(256), 0, st, th, count, seed,
+             index_base, coef_dev);
+  return QZO_OK;
+}
+int launch_update_vectors(float* const* table, const unsigned long long* base_table, int n_vec, int d, uint64_t seed,
+                          const float* coef_dev, cudaStream_t st) {
+  if (n_vec == 0) return QZO_OK;
+  if (d % 4) return QZO_ERR_BAD_ARG;
+  QZO_LAUNCH(update_vectors_kernel, dim3(ceil_div(d / 4, 256), n_vec), dim3(256), 0, st, table, base_table, d, seed, coef_dev);
+  return QZO_OK;
+}
+
 int launch_philox_words(uint64_t seed, uint64_t block_base, int64_t n_blocks, uint32_t* d_words,
                         float* d_uniforms, cudaStream_t st) {
   if (n_blocks == 0) return QZO_OK;

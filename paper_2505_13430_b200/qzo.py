@@ -28,6 +28,7 @@ EXPORTS = (
     "qzo_update_scales", "qzo_step", "qzo_step_host", "qzo_debug_set_capture", "qzo_debug_layer_output",
     "qzo_device_status", "qzo_launch_count", "qzo_profile_gemms", "qzo_profile_read",
     "qzo_step_begin", "qzo_step_finish", "qzo_get_scales", "qzo_set_scales", "qzo_debug_set_status",
+    "qzo_joint_workspace_bytes", "qzo_enable_joint_spsa",
 )
 
 
@@ -89,6 +90,8 @@ def _load():
         "qzo_get_scales": (ci, [vp, ci, vp, sz]),
         "qzo_set_scales": (ci, [vp, ci, vp, sz]),
         "qzo_debug_set_status": (ci, [vp, ci]),
+        "qzo_joint_workspace_bytes": (ci, [P(ModelDesc), P(sz)]),
+        "qzo_enable_joint_spsa": (ci, [vp, vp, sz, cf]),
         "qzo_debug_set_capture": (ci, [vp, ci]),
         "qzo_debug_layer_output": (ci, [vp, ci, ci, vp, sz]),
         "qzo_device_status": (ci, [vp, P(ci)]),
@@ -342,6 +345,20 @@ class Model:
     def qzo_set_scales(self, linear_id, values):
         _cuda(values, torch.bfloat16)
         _check(_lib.qzo_set_scales(self.handle, linear_id, _ptr(values), values.numel() * 2), "qzo_set_scales")
+
+    def qzo_enable_joint_spsa(self, lr_dense, on=True):
+        """Joint mode: embed, lm_head and the norm vectors are perturbed and updated too (plain SPSA)."""
+        if not on:
+            _check(_lib.qzo_enable_joint_spsa(self.handle, None, 0, 0.0), "qzo_enable_joint_spsa")
+            return
+        need = ctypes.c_size_t(0)
+        _check(_lib.qzo_joint_workspace_bytes(ctypes.byref(self.desc), ctypes.byref(need)), "qzo_joint_workspace_bytes")
+        self._joint_ws = torch.empty((need.value,), dtype=torch.uint8, device="cuda")
+        _check(_lib.qzo_enable_joint_spsa(self.handle, _ptr(self._joint_ws), need.value, lr_dense), "qzo_enable_joint_spsa")
+
+    def tensor(self, name):
+        """The caller-owned device tensor bound under `name` at construction (e.g. "embed", "L0.norm1_w")."""
+        return self._keep[name]
 
     def qzo_debug_set_status(self, value):
         _check(_lib.qzo_debug_set_status(self.handle, value), "qzo_debug_set_status")
