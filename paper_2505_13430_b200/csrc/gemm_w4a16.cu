@@ -61,6 +61,9 @@ constexpr int kSmemBudget = 227 * 1024;
 
 constexpr int kWTileBytes = kTileN * kBlockK * 2;      // 16 KiB bf16 A tile (bf16-weight path)
 constexpr int kCookedScaleBytes = kTileN * 8;          // {hi,hi},{lo,lo} per output feature
+constexpr int kRawScaleBytes = kTileN * 2;             // the group's stored bf16 scales of the tile's features
+// one slot of the nibble ring (int4 path): a quantisation group's packed nibbles, its perturbed scales, its stored scales
+constexpr int kNibSlotBytes = 2 * kPackedTileBytes + kCookedScaleBytes + kRawScaleBytes;
 
 enum OutMode { kOutBf16 = 0, kOutF32 = 1 };
 
@@ -313,7 +316,7 @@ struct SmemPlan {
   // three staging buffers: a pass waits for the TMA store issued two passes earlier, not for the last one
   static constexpr int kStagingBufs = 3;
   static constexpr int kStagingBytes = OUT_MODE == kOutBf16 ? kStagingBufs * kStagingBufBytes : 0;
-  static constexpr int kFixedBytes = kStagingBytes + kMaxASlots * kCookedScaleBytes + 1024 + 1024;
+  static constexpr int kFixedBytes = kStagingBytes + 1024 + 1024;
   // int4 path: the A ring (4 KiB of nibbles + 32 TMEM columns per stage) is as deep as tensor memory
   // allows, the B ring takes the shared memory that is left; bf16 path: both rings alike
   static constexpr int kStagesTmem = (512 - kAccCols) / kATmemColsPerStage;
@@ -325,15 +328,29 @@ struct SmemPlan {
   // Token tiles up to 128: the B ring also works in slots of two k-blocks (one wait, one expect and one
   // commit per quantisation group); there the per-k-block cost of the single-thread roles is the limit
   static constexpr int kBGroup = (DEQUANT && TOK <= 128) ? 2 : 1;
-  static constexpr int kBStages = DEQUANT ? cmin(8, (kSmemBudget - kFixedBytes - kAStages * kAStageBytes) / kXTileBytes) / kBGroup * kBGroup : 4;
+  // bytes of one slot of the ring that the A producer fills: int4 path: nibbles and scales of a group (the
+  // de-quantised operand lives in tensor memory); bf16 path: the 16 KiB tile the MMA reads
+  static constexpr int kNibBytes = DEQUANT ? kNibSlotBytes : kAStageBytes;
+  static constexpr int kBStages = DEQUANT ? cmin(8, (kSmemBudget - kFixedBytes - kASlots * kNibBytes) / kXTileBytes) / kBGroup * kBGroup : 4;
   static constexpr int kBSlots = kBStages / kBGroup;
   static_assert(kBSlots >= 2 && kASlots >= 2, "pipelines need at least two stages");
+  // int4 path: the nibble ring is deeper than the tensor-memory stages wherever shared memory is left (small
+  // token tiles): its slots are released as soon as the de-quantisers have read them, so the copies in
+  // flight, not the de-quantise / MMA / commit round of a tensor-memory stage, cover the HBM latency
+  static constexpr int kNibCap = TOK <= 64 ? 16 : 8;
+  // Token tiles up to 128: the stored scales of a group travel with its nibbles (a second bulk copy into the
+  // slot), so that the scale warps never wait for a load from HBM.  256-token tiles keep the scale warps'
+  // own early load: there the ring has four slots, and the perturbed scales must be written the moment a
+  // slot is released.
+  static constexpr bool kRawViaCopy = DEQUANT && TOK <= 128;
+  static constexpr int kNibLeft = (kSmemBudget - kFixedBytes - kBStages * kXTileBytes - 3 * 8 * 16 - 64) / kNibBytes;
+  static constexpr int kNibSlots = DEQUANT ? (kNibLeft < kASlots ? kASlots : cmin(kNibCap, kNibLeft)) : kASlots;
+  static_assert(kNibSlots >= kASlots, "nibble ring at least as deep as the tensor-memory stages");
   static constexpr int kOffB = 0;
-  static constexpr int kOffA = kBStages * kXTileBytes;
-  static constexpr int kOffStaging = kOffA + kAStages * kAStageBytes;
-  static constexpr int kOffCooked = kOffStaging + kStagingBytes;
-  static constexpr int kOffBars = kOffCooked + kMaxASlots * kCookedScaleBytes;
-  static constexpr int kNumBars = 2 * kBStages + 3 * kAStages + 2;
+  static constexpr int kOffA = kBStages * kXTileBytes;                 // nibble ring / bf16 A ring
+  static constexpr int kOffStaging = kOffA + kNibSlots * kNibBytes;
+  static constexpr int kOffBars = kOffStaging + kStagingBytes;
+  static constexpr int kNumBars = 2 * kBStages + 3 * kNibSlots + 2 * kAStages + 2;
   static constexpr int kOffMisc = kOffBars + kNumBars * 8;
   static constexpr int kTotal = kOffMisc + 32;
   static constexpr int kDynamicBytes = kTotal + 1024;      // slack for the 1024-byte alignment
@@ -402,10 +419,17 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
   const uint32_t bar0 = base + Plan::kOffBars;
   auto bar_b_full = [&](int s) { return bar0 + 8u * s; };                        // activation tile landed
   auto bar_b_empty = [&](int s) { return bar0 + 8u * (kBStages + s); };          // MMAs that read it retired
-  auto bar_a_full = [&](int s) { return bar0 + 8u * (2 * kBStages + s); };       // packed nibbles / bf16 weights landed
-  auto bar_a_deq = [&](int s) { return bar0 + 8u * (2 * kBStages + kAStages + s); };      // A stage de-quantised
-  auto bar_a_empty = [&](int s) { return bar0 + 8u * (2 * kBStages + 2 * kAStages + s); };  // MMAs that read it retired
-  const uint32_t bar_acc_full = bar0 + 8u * (2 * kBStages + 3 * kAStages);       // accumulator complete
+  constexpr int kNibSlots = Plan::kNibSlots;
+  // nibble ring (int4 path) / A ring (bf16 path): full = nibbles landed and perturbed scales written (bf16
+  // path: unused, the B barrier counts both tiles); raw = the group's stored scales landed; free = the
+  // de-quantisers have read the slot (bf16 path: the MMAs that read it retired)
+  auto bar_nib_full = [&](int s) { return bar0 + 8u * (2 * kBStages + s); };
+  auto bar_nib_raw = [&](int s) { return bar0 + 8u * (2 * kBStages + kNibSlots + s); };
+  auto bar_nib_free = [&](int s) { return bar0 + 8u * (2 * kBStages + 2 * kNibSlots + s); };
+  // tensor-memory stages of the de-quantised operand (one slot = one group = two k-blocks)
+  auto bar_a_deq = [&](int s) { return bar0 + 8u * (2 * kBStages + 3 * kNibSlots + s); };                // de-quantised
+  auto bar_a_empty = [&](int s) { return bar0 + 8u * (2 * kBStages + 3 * kNibSlots + kAStages + s); };   // MMAs that read it retired
+  const uint32_t bar_acc_full = bar0 + 8u * (2 * kBStages + 3 * kNibSlots + 2 * kAStages);   // accumulator complete
   const uint32_t bar_acc_empty = bar_acc_full + 8u;                              // accumulator drained
   volatile int* const abort_flag = reinterpret_cast<volatile int*>(smem + Plan::kOffMisc);
   uint32_t* const tmem_slot = reinterpret_cast<uint32_t*>(smem + Plan::kOffMisc + 4);
@@ -432,10 +456,14 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
       mbar_init(bar_b_full(s), DEQUANT ? 1 : 2);
       mbar_init(bar_b_empty(s), 1);
     }
-    for (int s = 0; s < kASlots; ++s) {
+    for (int s = 0; s < kNibSlots; ++s) {
       // int4 path: the slot is full when its nibbles have landed AND its perturbed scales are written
-      mbar_init(bar_a_full(s), DEQUANT ? 2 : 1);
-      mbar_init(bar_a_deq(s), kNumDeqWarps / 2);        // one team of four de-quantiser warps per group
+      mbar_init(bar_nib_full(s), DEQUANT ? 2 : 1);
+      mbar_init(bar_nib_raw(s), 1);
+      mbar_init(bar_nib_free(s), DEQUANT ? kNumDeqWarps / 2 : 1);   // one team of four de-quantiser warps per group
+    }
+    for (int s = 0; s < kASlots; ++s) {
+      mbar_init(bar_a_deq(s), kNumDeqWarps / 2);
       mbar_init(bar_a_empty(s), 1);
     }
     mbar_init(bar_acc_full, 1);
@@ -458,7 +486,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     // warp 0 feeds the B ring (activation tiles), warp 2 the A ring (packed nibbles / bf16 weights)
     if (lane == 0) {
       const bool is_b = warp == 0;
-      const int stages = is_b ? kBSlots : kASlots;
+      const int stages = is_b ? kBSlots : kNibSlots;
       Ring ring;
       int issued = 0;
       for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x) {
@@ -479,12 +507,20 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
           for (int it = 0; it < w.nkb; it += kAGroup) {
             const int kb = w.kb_begin + it;
             const int nk = min(kAGroup, w.nkb - it);         // k-blocks of this slot (the last group of an odd K has one)
-            if (!mbar_wait(bar_a_empty(ring.s), ring.ph ^ 1u, abort_flag)) { ok = false; break; }
-            const uint32_t dst = base + Plan::kOffA + ring.s * (kAGroup * Plan::kAStageBytes);
+            if (!mbar_wait(bar_nib_free(ring.s), ring.ph ^ 1u, abort_flag)) { ok = false; break; }
+            const uint32_t dst = base + Plan::kOffA + ring.s * Plan::kNibBytes;
             if (DEQUANT) {
-              mbar_arrive_expect_tx(bar_a_full(ring.s), (uint32_t)(nk * kPackedTileBytes));
+              mbar_arrive_expect_tx(bar_nib_full(ring.s), (uint32_t)(nk * kPackedTileBytes));
               bulk_load(dst, L.wq + ((size_t)(w.n0 / kTileN) * p.num_kb + kb) * kPackedTileBytes,
-                        (uint32_t)(nk * kPackedTileBytes), bar_a_full(ring.s));
+                        (uint32_t)(nk * kPackedTileBytes), bar_nib_full(ring.s));
+              // the group's stored scales of this tile's features travel with the nibbles (N is a multiple of 8
+              // and the scale rows are 16-byte aligned, so is every run of them)
+              if (Plan::kRawViaCopy) {
+                const uint32_t raw_bytes = (uint32_t)min(kTileN, L.N - w.n0) * 2u;
+                mbar_arrive_expect_tx(bar_nib_raw(ring.s), raw_bytes);
+                bulk_load(dst + 2 * kPackedTileBytes + kCookedScaleBytes, L.scales + (size_t)(kb >> 1) * L.N + w.n0, raw_bytes,
+                          bar_nib_raw(ring.s));
+              }
             } else {
               mbar_arrive_expect_tx(bar_b_full(ring.s), Plan::kAStageBytes);
               tma_load_2d(dst, &tmap_w, bar_b_full(ring.s), kb * kBlockK, w.n0);
@@ -500,9 +536,14 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         const int pending = min(issued, stages);
         for (int j = 0; j < pending; ++j) {
           const int idx = issued - 1 - j;
-          const uint32_t bar = (is_b || !DEQUANT) ? bar_b_full(idx % stages) : bar_a_full(idx % stages);
+          // int4 path: the slot's "full" barrier also counts a scale warp, which may have given up; its copies
+          // are waited for through the stored scales' barrier (issued last) where there is one
+          const uint32_t bar = (is_b || !DEQUANT) ? bar_b_full(idx % stages)
+                                                  : (Plan::kRawViaCopy ? bar_nib_raw(idx % stages) : bar_nib_full(idx % stages));
           mbar_wait(bar, (uint32_t)(idx / stages) & 1u, never_set);
         }
+        // a nibble copy issued just before an awaited scale copy may land a moment after it
+        if (!is_b && Plan::kRawViaCopy) __nanosleep(50000);
       }
     }
   } else if (warp == 1) {
@@ -541,14 +582,14 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             static_assert(kBlockK == 64, "four K = 16 steps per k-block");
             umma_bf16_tmem_a_x4(tmem_d, a_tmem, bdesc, idesc, it > 0 ? 1u : 0u);
           } else {
-            const uint64_t adesc = umma_desc_k_major_sw128(base + Plan::kOffA + ra.s * Plan::kAStageBytes);
+            const uint64_t adesc = umma_desc_k_major_sw128(base + Plan::kOffA + ra.s * Plan::kNibBytes);
 #pragma unroll
             for (int k = 0; k < kBlockK / 16; ++k)
               umma_bf16(tmem_d, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
                         (it > 0 || k > 0) ? 1u : 0u);
           }
           if (bslot_done) umma_commit(bar_b_empty(rb.s)); // releases the B slot
-          if (slot_done) umma_commit(bar_a_empty(ra.s));  // and, after its last k-block, the A slot
+          if (slot_done) umma_commit(DEQUANT ? bar_a_empty(ra.s) : bar_nib_free(ra.s));  // and, after its last k-block, the A slot
         }
         if (slot_done) ra.next(kASlots);
         if (bslot_done) rb.next(kBSlots);
@@ -596,25 +637,36 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         const int ngroups = (w.nkb + 1) >> 1;
         for (int gi = 0; gi < ngroups; ++gi, ++gig) {
           if ((gig % kNumScaleWarps) != sw) continue;
-          const int slot = gig % kASlots;                // the A-ring slot of this group
-          const uint32_t gph = (uint32_t)(gig / kASlots) & 1u;
+          const int slot = gig % kNibSlots;              // the nibble-ring slot of this group
+          const uint32_t gph = (uint32_t)(gig / kNibSlots) & 1u;
           const int g = (w.kb_begin >> 1) + gi;
           const int r0 = lane * 4;                       // four consecutive output features = one counter block
+          const bool live = w.n0 + r0 < L.N;             // N is a multiple of 8: all four or none
+          // z does not depend on the stored scales: it is ready before they land
+          float z[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+          float se = 0.0f;
+          if (live && p.sign_eps != 0.0f) {
+            const uint64_t i0 = L.idx_base + (uint64_t)g * (uint64_t)L.N + (uint64_t)(w.n0 + r0);
+            normals_of_block(p.seed, i0 >> 2, z);
+            // token tiles never straddle pair_rows (checked on the host)
+            se = (p.pair_rows > 0 && w.tok0 >= p.pair_rows) ? -p.sign_eps : p.sign_eps;
+          }
+          uint8_t* const slot_mem = smem + Plan::kOffA + slot * Plan::kNibBytes;
+          uint2 raw = make_uint2(0u, 0u);
+          if (!Plan::kRawViaCopy && live) raw = *reinterpret_cast<const uint2*>(L.scales + (size_t)g * L.N + w.n0 + r0);
+          // kRawViaCopy: the stored scales came with the nibbles' copy; their arrival also says that the slot was
+          // free.  Otherwise: the slot is free once the de-quantisers have read its previous group.
+          const bool got = Plan::kRawViaCopy ? mbar_wait_relaxed(bar_nib_raw(slot), gph, abort_flag)
+                                             : mbar_wait_relaxed(bar_nib_free(slot), gph ^ 1u, abort_flag);
+          if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
           float sv[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-          if (w.n0 + r0 < L.N) {                         // N is a multiple of 8: all four or none
-            const uint2 raw = *reinterpret_cast<const uint2*>(L.scales + (size_t)g * L.N + w.n0 + r0);
+          if (live) {
+            if (Plan::kRawViaCopy)
+              raw = *reinterpret_cast<const uint2*>(slot_mem + 2 * kPackedTileBytes + kCookedScaleBytes + r0 * 2);
             const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
             const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
-            sv[0] = __low2float(a); sv[1] = __high2float(a); sv[2] = __low2float(b); sv[3] = __high2float(b);
-            if (p.sign_eps != 0.0f) {
-              float z[4];
-              const uint64_t i0 = L.idx_base + (uint64_t)g * (uint64_t)L.N + (uint64_t)(w.n0 + r0);
-              normals_of_block(p.seed, i0 >> 2, z);
-              // token tiles never straddle pair_rows (checked on the host)
-              const float se = (p.pair_rows > 0 && w.tok0 >= p.pair_rows) ? -p.sign_eps : p.sign_eps;
-#pragma unroll
-              for (int l = 0; l < 4; ++l) sv[l] = fmaf(se, z[l], sv[l]);
-            }
+            sv[0] = fmaf(se, z[0], __low2float(a)); sv[1] = fmaf(se, z[1], __high2float(a));
+            sv[2] = fmaf(se, z[2], __low2float(b)); sv[3] = fmaf(se, z[3], __high2float(b));
           }
           uint32_t cooked[8];
 #pragma unroll
@@ -625,13 +677,11 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             cooked[2 * l] = h16 | (h16 << 16);
             cooked[2 * l + 1] = l16 | (l16 << 16);
           }
-          // the slot (nibbles, scales, tensor-memory stages) is free once the MMAs of its previous group retired
-          if (!__all_sync(0xffffffffu, mbar_wait_relaxed(bar_a_empty(slot), gph ^ 1u, abort_flag))) { ok = false; break; }
-          uint4* dst = reinterpret_cast<uint4*>(smem + Plan::kOffCooked + slot * kCookedScaleBytes + r0 * 8);
+          uint4* dst = reinterpret_cast<uint4*>(slot_mem + 2 * kPackedTileBytes + r0 * 8);
           dst[0] = make_uint4(cooked[0], cooked[1], cooked[2], cooked[3]);
           dst[1] = make_uint4(cooked[4], cooked[5], cooked[6], cooked[7]);
           __syncwarp();
-          if (lane == 0) mbar_arrive(bar_a_full(slot));
+          if (lane == 0) mbar_arrive(bar_nib_full(slot));
         }
       }
       if (!ok) *abort_flag = 1;
@@ -667,27 +717,34 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         const Unit w = decode_unit(p, u, TOK);
         for (int it = 0; it < w.nkb; it += 2, ++gig) {
           if ((gig & 1) != team) continue;                    // the other team's group
-          const int slot = gig % kASlots;                     // A-ring slot = one quantisation group (two k-blocks)
+          const int nslot = gig % kNibSlots;                  // nibble-ring slot of this group
+          const uint32_t nph = (uint32_t)(gig / kNibSlots) & 1u;
+          const int slot = gig % kASlots;                     // tensor-memory slot = one quantisation group (two k-blocks)
           const uint32_t gph = (uint32_t)(gig / kASlots) & 1u;
           const bool two = it + 1 < w.nkb;                    // the last group of an odd K has one k-block
-          // the slot is full: nibbles landed, perturbed scales written; that implies it had been released
-          // by the MMAs that last read it
-          if (!__all_sync(0xffffffffu, mbar_wait(bar_a_full(slot), gph, abort_flag))) { ok = false; break; }
+          // the nibble slot is full: nibbles landed, perturbed scales written
+          if (!__all_sync(0xffffffffu, mbar_wait(bar_nib_full(nslot), nph, abort_flag))) { ok = false; break; }
+          const uint8_t* const slot_mem = smem + Plan::kOffA + nslot * Plan::kNibBytes;
           {
-            const uint2 c = *reinterpret_cast<const uint2*>(smem + Plan::kOffCooked + slot * kCookedScaleBytes + r * 8);
+            const uint2 c = *reinterpret_cast<const uint2*>(slot_mem + 2 * kPackedTileBytes + r * 8);
             *reinterpret_cast<uint32_t*>(&s_hi) = c.x;
             *reinterpret_cast<uint32_t*>(&s_lo) = c.y;
           }
           // this row's 64 k of each k-block: two 16-byte units (32 k each)
-          const uint8_t* src = smem + Plan::kOffA + slot * (2 * Plan::kAStageBytes) + r * 16;
+          const uint8_t* src = slot_mem + r * 16;
           uint4 pk[4];
           pk[0] = *reinterpret_cast<const uint4*>(src);
           pk[1] = *reinterpret_cast<const uint4*>(src + kTileN * 16);
           pk[2] = pk[3] = make_uint4(0, 0, 0, 0);
           if (two) {
-            pk[2] = *reinterpret_cast<const uint4*>(src + Plan::kAStageBytes);
-            pk[3] = *reinterpret_cast<const uint4*>(src + Plan::kAStageBytes + kTileN * 16);
+            pk[2] = *reinterpret_cast<const uint4*>(src + kPackedTileBytes);
+            pk[3] = *reinterpret_cast<const uint4*>(src + kPackedTileBytes + kTileN * 16);
           }
+          // the slot's bytes are in registers: hand it back to the producer at once
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_nib_free(nslot));
+          // the tensor-memory stages of the slot are free once the MMAs of their previous group retired
+          if (!__all_sync(0xffffffffu, mbar_wait(bar_a_empty(slot), gph ^ 1u, abort_flag))) { ok = false; break; }
           tcgen05_fence_after();                              // orders the MMAs' reads of this slot before the stores below
           uint32_t outw[16];
 #pragma unroll

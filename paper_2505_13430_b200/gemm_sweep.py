@@ -22,6 +22,7 @@ from . import inputs, qzo
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 L2_BYTES = 126 * 2 ** 20
+NOMINAL_HBM_GBS, NOMINAL_BF16_TFLOPS = 8000.0, 2250.0      # datasheet figures, for the second column
 
 
 def peaks():
@@ -118,10 +119,18 @@ def main():
                          "frac": roof / us, "tflops": 2.0 * M * K * N / us / 1e6, "gbs": gemm_bytes(M, K, N) / us / 1e3,
                          "best_pass_us": best_us, "rotation_sets": n_sets})
             r = rows[-1]
+            roof_nom = max(gemm_bytes(M, K, N) / (NOMINAL_HBM_GBS * 1e9), 2.0 * M * K * N / (NOMINAL_BF16_TFLOPS * 1e12)) * 1e6
+            r["frac_of_nominal"] = roof_nom / us
+            r["splits"] = qzo.qzo_gemm_workspace_bytes(M, K, N) // (M * N * 4)
             if not args.json:
                 print(f"K={K:6d} N={N:6d} M={M:5d}  {us:9.2f} us  roofline {roof:8.2f} us ({r['bound']:6s})  "
-                      f"frac {r['frac']:.3f}  {r['tflops']:8.1f} TFLOP/s  {r['gbs']:8.1f} GB/s  best pass {best_us:8.2f} us  sets={n_sets}",
+                      f"frac {r['frac']:.3f} (of nominal peaks {r['frac_of_nominal']:.3f})  {r['tflops']:8.1f} TFLOP/s  "
+                      f"{r['gbs']:8.1f} GB/s  best pass {best_us:8.2f} us  K slices {max(r['splits'], 1)}  sets={n_sets}",
                       flush=True)
+    if not args.json:
+        print(f"peaks ({src}): HBM {bw:.1f} GB/s, dense bf16 {tf:.1f} TFLOP/s; nominal: {NOMINAL_HBM_GBS:.0f} GB/s, "
+              f"{NOMINAL_BF16_TFLOPS:.0f} TFLOP/s; min frac {min(r['frac'] for r in rows):.3f}, "
+              f"rows at or above 0.70: {sum(r['frac'] >= 0.70 for r in rows)} of {len(rows)}")
     if args.json:
         print(json.dumps({"peaks": {"hbm_gbs": bw, "bf16_tflops": tf, "source": src}, "rows": rows}))
 
