@@ -3,6 +3,11 @@
 Eq. 5 perturbs only the scales: Delta' = Delta + sign * eps * z, the integer
 weights stay fixed; Eq. 4 then gives the weight Delta' * w_bar that the normal
 forward uses.  No clamp is applied to Delta' (Algorithm 1, PERTURB_SCALES).
+
+The same estimator applies to block-scaled codebook formats (the paper's NF4
+experiment, appendix "Results with Stable Diffusion": the continuous scales of a
+4-bit codebook quantiser are what QZO perturbs and updates): there the fixed part
+of a weight is a table entry instead of an integer, see perturbed_linear_table16.
 """
 import numpy as np
 from . import philox
@@ -50,4 +55,26 @@ def perturbed_linear_samples(x_rows, q_cols, s_cols, cols, N, seed, index_base, 
     y = x @ w
     if bias_cols is not None:
         y = y + np.asarray(bias_cols, dtype=np.float64)[None, :]
+    return y
+
+
+TABLE_BLOCK = 64
+
+
+def perturbed_linear_table16(x, codes, s, table, seed, index_base, sign, eps, bias=None):
+    """Block-scaled 16-entry codebook weights (NF4-style storage): w[k][n] = s'[k // 64][n] * table[codes[k][n]],
+    codes in [0, 15], one scale per block of 64 consecutive input rows of an output column, and
+    s' = s + sign*eps*z with z at index index_base + b*N + n for scale [b][n] (Eq. 5 on the format's
+    continuous scales; the codes and the table stay fixed).  Y = X W (+ bias), fp64."""
+    x = np.asarray(x, dtype=np.float64)
+    codes = np.asarray(codes)
+    table = np.asarray(table, dtype=np.float64)
+    assert table.shape == (16,) and codes.min() >= 0 and codes.max() <= 15
+    K = codes.shape[0]
+    sp = perturbed_scales(s, seed, index_base, sign, eps)
+    assert sp.shape[0] == (K + TABLE_BLOCK - 1) // TABLE_BLOCK
+    w = sp[np.arange(K) // TABLE_BLOCK] * table[codes]
+    y = x @ w
+    if bias is not None:
+        y = y + np.asarray(bias, dtype=np.float64)[None, :]
     return y

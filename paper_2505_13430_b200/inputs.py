@@ -125,3 +125,18 @@ def gemm_case(M, K, N, seed=0, device="cpu"):
     s = (torch.rand((G, N), generator=g, dtype=torch.float32, device=device) * 0.015
          + 0.005).bfloat16()
     return x, q, s
+
+
+def table16_case(M, K, N, seed=0, device="cpu"):
+    """Inputs of the block-scaled 16-entry-codebook GEMM (NF4-style storage): X bf16 ~ N(0,1) [M][K]; codes
+    int8 uniform in [0,15] [K][N]; scales bf16 uniform in [0.01, 0.04] [ceil(K/64)][N] (absmax-like: the
+    table lies in [-1, 1]); table = 16 increasing fp32 values in [-1, 1] drawn from the seed (sorted uniform
+    draws with the end points pinned to -1 and 1), standing in for a trained or published codebook."""
+    g = _gen(seed, device)
+    x = torch.randn((M, K), generator=g, dtype=torch.float32, device=device).bfloat16()
+    codes = torch.randint(0, 16, (K, N), generator=g, dtype=torch.int8, device=device)
+    B = (K + 63) // 64
+    s = (torch.rand((B, N), generator=g, dtype=torch.float32, device=device) * 0.03 + 0.01).bfloat16()
+    t = torch.sort(torch.rand((16,), generator=g, dtype=torch.float32, device=device) * 2.0 - 1.0).values
+    t[0], t[15] = -1.0, 1.0
+    return x, codes, s, t

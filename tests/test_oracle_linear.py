@@ -76,3 +76,36 @@ def test_sampled_columns_equal_the_full_layer():
         acc += x[t, k] * (float(s[g, n]) + eps * z) * int(q[k, n])
     got = linear.perturbed_linear_samples(x[[t]], q[:, [n]], s[:, [n]], [n], 24, seed, base, +1, eps)[0, 0]
     assert abs(acc - got) <= 1e-12 * max(1.0, abs(acc))
+
+
+def test_table16_linear_brute_force_and_special_cases():
+    # block-scaled 16-entry codebook weights: triple loop on a small case, sign 0 = plain de-quantised GEMM,
+    # the two linearity identities of the perturbation, and the reduction to the int4 routine
+    from paper_2505_13430_b200 import inputs
+    x, codes, s, table = inputs.table16_case(3, 136, 16, seed=2)
+    x, codes, s, table = x.float().numpy(), codes.numpy(), s.float().numpy(), table.numpy()
+    seed, base, eps = 5, 32, 2e-3
+    z = philox.normal_range(seed, base, s.size).astype(np.float64).reshape(s.shape)
+    for sign in (+1, -1, 0):
+        got = linear.perturbed_linear_table16(x, codes, s, table, seed, base, sign, eps)
+        want = np.zeros((3, 16))
+        for t in range(3):
+            for n in range(16):
+                for k in range(136):
+                    want[t, n] += float(x[t, k]) * (float(s[k // 64, n]) + sign * eps * z[k // 64, n]) * float(table[codes[k, n]])
+        assert np.abs(got - want).max() <= 1e-12 * np.abs(want).max()
+    y0 = linear.perturbed_linear_table16(x, codes, s, table, seed, base, 0, eps)
+    yp = linear.perturbed_linear_table16(x, codes, s, table, seed, base, +1, eps)
+    ym = linear.perturbed_linear_table16(x, codes, s, table, seed, base, -1, eps)
+    assert np.abs(yp + ym - 2 * y0).max() <= 1e-12 * np.abs(y0).max()
+    zt = z[np.arange(136) // 64] * table.astype(np.float64)[codes]
+    assert np.abs((yp - ym) - 2 * eps * (x.astype(np.float64) @ zt)).max() <= 1e-12 * np.abs(yp - ym).max()
+    # with the affine table c - 8 and equal scales in the two blocks of every group it IS the int4 linear
+    K, N = 256, 8
+    rng = np.random.default_rng(3)
+    xx = rng.standard_normal((4, K))
+    q = rng.integers(-8, 8, size=(K, N)).astype(np.int8)
+    s128 = int4.bf16_round(rng.uniform(0.005, 0.02, size=(2, N)).astype(np.float32))
+    a = linear.perturbed_linear(xx, q, s128, 1, 0, 0, 1e-3)
+    b = linear.perturbed_linear_table16(xx, q + 8, np.repeat(s128, 2, axis=0), np.arange(16) - 8.0, 1, 0, 0, 1e-3)
+    assert np.abs(a - b).max() <= 1e-13 * np.abs(a).max()
