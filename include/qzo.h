@@ -108,6 +108,20 @@ int qzo_perturbed_gemm(const void* d_x_bf16, const void* d_wq, const void* d_sca
                        uint64_t seed, uint64_t scale_index_base, int sign, float eps,
                        void* d_workspace, size_t workspace_bytes, int* d_status, void* stream);
 
+/* The same linear for weights stored as 4-bit codes into a 16-entry table with one scale per block of 64
+ * rows (block-scaled codebook storage such as NF4; the paper applies QZO to NF4 weights in its appendix
+ * "Results with Stable Diffusion" and to codebook weights with channel-wise scales in Sec. 4.1: what QZO
+ * perturbs and updates is the format's continuous scale, Eq. 5, so only the de-quantisation prologue differs):
+ *   Y[t][n] = sum_k X[t][k] (s[k/64][n] + sign eps z_i) table[c[k][n]] (+ bias[n]),  i = scale_index_base + (k/64) N + n.
+ * d_codes: codes c in [0, 15] in the kernel layout of qzo_repack_int4 (pack them like int4 values, code =
+ * stored nibble); d_scales bf16 [ceil(K/64)][N]; h_table16: HOST pointer to the 16 table values (read during
+ * the call, rounded to bf16 on the device).  Everything else as qzo_perturbed_gemm; the seeded update of such
+ * scales is qzo_update_scales_flat. */
+int qzo_perturbed_gemm_table16(const void* d_x_bf16, const void* d_codes, const void* d_scales_bf16,
+                               const float* h_table16, const float* d_bias, void* d_y_bf16, int M, int K, int N,
+                               uint64_t seed, uint64_t scale_index_base, int sign, float eps,
+                               void* d_workspace, size_t workspace_bytes, int* d_status, void* stream);
+
 /* The same linear for callers that must not allocate device memory and have no workspace to
  * lend: for example a serving process that gave all device memory to its own pool when it
  * started, or a latency-critical loop in which the device-wide synchronisation of an allocation

@@ -37,6 +37,7 @@
 #include "layers.cuh"
 
 #include <cuda.h>
+#include <cstring>
 #include <mutex>
 
 namespace qzo {
@@ -61,9 +62,16 @@ constexpr int kSmemBudget = 227 * 1024;
 
 constexpr int kWTileBytes = kTileN * kBlockK * 2;      // 16 KiB bf16 A tile (bf16-weight path)
 constexpr int kCookedScaleBytes = kTileN * 8;          // {hi,hi},{lo,lo} per output feature
-constexpr int kRawScaleBytes = kTileN * 2;             // the group's stored bf16 scales of the tile's features
-// one slot of the nibble ring (int4 path): a quantisation group's packed nibbles, its perturbed scales, its stored scales
-constexpr int kNibSlotBytes = 2 * kPackedTileBytes + kCookedScaleBytes + kRawScaleBytes;
+constexpr int kRawScaleBytes = kTileN * 2;             // one row of stored bf16 scales of the tile's features
+constexpr int kLutSmemBytes = 16 * 32 * 4;             // table mode: every codebook value as a bf16 pair, one copy per lane (bank)
+
+// How the A operand comes about.
+enum WeightMode {
+  kWBf16 = 0,     // bf16 [N][K] matrix loaded as it is (lm_head)
+  kWInt4 = 1,     // packed int4, one scale per group of 128 k: w = (u - 8) s'   (Eq. 4, the paper's GPTQ setting)
+  kWTable16 = 2   // packed 4-bit codes into a 16-entry table, one scale per block of 64 k: w = table[u] s'
+                  // (block-scaled codebook storage such as NF4; only the prologue differs)
+};
 
 enum OutMode { kOutBf16 = 0, kOutF32 = 1 };
 
@@ -88,6 +96,7 @@ struct GemmParams {
   float sign_eps;                 // sign * eps (0 when unperturbed)
   int pair_rows;                  // > 0: token rows from this one on take -sign_eps (both passes of a step in one launch)
   int* status;
+  float lut[16];                  // table mode: the 16 codebook values (a nibble is an index into them)
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -304,8 +313,15 @@ constexpr int cmin(int a, int b) { return a < b ? a : b; }
 // tensor memory) is deep and cheap, so the de-quantisers run well ahead of the tensor pipe; the
 // B ring holds the activation tiles.  A finished bf16 tile leaves in passes of up to 32 tokens
 // through three staging buffers, each pass as one TMA store.
-template <int TOK, bool DEQUANT, int OUT_MODE>
+template <int TOK, int WMODE, int OUT_MODE>
 struct SmemPlan {
+  static constexpr bool DEQUANT = WMODE != kWBf16;
+  static constexpr bool LUT = WMODE == kWTable16;
+  static constexpr int kScaleRows = LUT ? 2 : 1;       // rows of scales per ring slot (a slot is 128 k)
+  // one slot of the nibble ring: a group's packed nibbles, its perturbed scales, its stored scales
+  static constexpr int kOffCookedInSlot = 2 * kPackedTileBytes;
+  static constexpr int kOffRawInSlot = kOffCookedInSlot + kScaleRows * kCookedScaleBytes;
+  static constexpr int kNibSlotBytes = kOffRawInSlot + kScaleRows * kRawScaleBytes;
   static constexpr int kAccCols = TOK < 32 ? 32 : TOK;
   static constexpr int kXTileBytes = TOK * kBlockK * 2;
   // int4 path: A stage = 4 KiB of packed nibbles; bf16 path: A stage = 16 KiB bf16 tile (read by the MMA)
@@ -316,7 +332,7 @@ struct SmemPlan {
   // three staging buffers: a pass waits for the TMA store issued two passes earlier, not for the last one
   static constexpr int kStagingBufs = 3;
   static constexpr int kStagingBytes = OUT_MODE == kOutBf16 ? kStagingBufs * kStagingBufBytes : 0;
-  static constexpr int kFixedBytes = kStagingBytes + 1024 + 1024;
+  static constexpr int kFixedBytes = kStagingBytes + 1024 + 1024 + (LUT ? kLutSmemBytes : 0);
   // int4 path: the A ring (4 KiB of nibbles + 32 TMEM columns per stage) is as deep as tensor memory
   // allows, the B ring takes the shared memory that is left; bf16 path: both rings alike
   static constexpr int kStagesTmem = (512 - kAccCols) / kATmemColsPerStage;
@@ -349,7 +365,8 @@ struct SmemPlan {
   static constexpr int kOffB = 0;
   static constexpr int kOffA = kBStages * kXTileBytes;                 // nibble ring / bf16 A ring
   static constexpr int kOffStaging = kOffA + kNibSlots * kNibBytes;
-  static constexpr int kOffBars = kOffStaging + kStagingBytes;
+  static constexpr int kOffLut = kOffStaging + kStagingBytes;
+  static constexpr int kOffBars = kOffLut + (LUT ? kLutSmemBytes : 0);
   static constexpr int kNumBars = 2 * kBStages + 3 * kNibSlots + 2 * kAStages + 2;
   static constexpr int kOffMisc = kOffBars + kNumBars * 8;
   static constexpr int kTotal = kOffMisc + 32;
@@ -393,14 +410,17 @@ struct Ring {
 };
 
 // ----------------------------------------------------------------------------- the kernel
-// DEQUANT = true : A operand produced from packed int4 + perturbed scales.
-// DEQUANT = false: A operand is a bf16 [N][K] row-major matrix loaded through tmap_w (lm_head).
-template <int TOK, bool DEQUANT, int OUT_MODE>
+// WMODE (WeightMode): kWInt4 / kWTable16: A operand produced from packed 4-bit codes + perturbed scales;
+// kWBf16: A operand is a bf16 [N][K] row-major matrix loaded through tmap_w (lm_head).
+template <int TOK, int WMODE, int OUT_MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                   const __grid_constant__ CUtensorMap tmap_y0, const __grid_constant__ CUtensorMap tmap_y1,
                   const __grid_constant__ CUtensorMap tmap_y2, const __grid_constant__ GemmParams p) {
-  using Plan = SmemPlan<TOK, DEQUANT, OUT_MODE>;
+  using Plan = SmemPlan<TOK, WMODE, OUT_MODE>;
+  constexpr bool DEQUANT = Plan::DEQUANT;
+  constexpr bool LUT = Plan::LUT;
+  constexpr int kScaleRows = Plan::kScaleRows;
   constexpr int kAStages = Plan::kAStages;
   constexpr int kASlots = Plan::kASlots;
   constexpr int kAGroup = Plan::kAGroup;
@@ -470,6 +490,11 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     mbar_init(bar_acc_empty, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  if (LUT && threadIdx.x < 512) {
+    // codebook value e as a bf16 pair {t, t}, one copy per lane: entry (e, lane) sits in bank `lane`
+    const uint32_t t16 = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(p.lut[threadIdx.x >> 5]));
+    reinterpret_cast<uint32_t*>(smem + Plan::kOffLut)[threadIdx.x] = t16 | (t16 << 16);
+  }
   if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
   tcgen05_fence_before();
   __syncthreads();
@@ -517,9 +542,13 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
               // and the scale rows are 16-byte aligned, so is every run of them)
               if (Plan::kRawViaCopy) {
                 const uint32_t raw_bytes = (uint32_t)min(kTileN, L.N - w.n0) * 2u;
-                mbar_arrive_expect_tx(bar_nib_raw(ring.s), raw_bytes);
-                bulk_load(dst + 2 * kPackedTileBytes + kCookedScaleBytes, L.scales + (size_t)(kb >> 1) * L.N + w.n0, raw_bytes,
-                          bar_nib_raw(ring.s));
+                // int4: the group's row of scales; table mode: one row per k-block of the slot
+                const int rows = LUT ? nk : 1;
+                const int row0 = LUT ? kb : (kb >> 1);
+                mbar_arrive_expect_tx(bar_nib_raw(ring.s), raw_bytes * (uint32_t)rows);
+                for (int j = 0; j < rows; ++j)
+                  bulk_load(dst + Plan::kOffRawInSlot + j * kRawScaleBytes, L.scales + (size_t)(row0 + j) * L.N + w.n0, raw_bytes,
+                            bar_nib_raw(ring.s));
               }
             } else {
               mbar_arrive_expect_tx(bar_b_full(ring.s), Plan::kAStageBytes);
@@ -639,47 +668,58 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
           if ((gig % kNumScaleWarps) != sw) continue;
           const int slot = gig % kNibSlots;              // the nibble-ring slot of this group
           const uint32_t gph = (uint32_t)(gig / kNibSlots) & 1u;
-          const int g = (w.kb_begin >> 1) + gi;
           const int r0 = lane * 4;                       // four consecutive output features = one counter block
           const bool live = w.n0 + r0 < L.N;             // N is a multiple of 8: all four or none
+          // rows of scales of this slot: int4: the group's row; table mode: one row per k-block (block of 64 k)
+          const int row0 = LUT ? w.kb_begin + 2 * gi : (w.kb_begin >> 1) + gi;
+          const int rows = LUT ? min(2, w.nkb - 2 * gi) : 1;
+          // token tiles never straddle pair_rows (checked on the host)
+          const float se = (p.pair_rows > 0 && w.tok0 >= p.pair_rows) ? -p.sign_eps : p.sign_eps;
           // z does not depend on the stored scales: it is ready before they land
-          float z[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-          float se = 0.0f;
-          if (live && p.sign_eps != 0.0f) {
-            const uint64_t i0 = L.idx_base + (uint64_t)g * (uint64_t)L.N + (uint64_t)(w.n0 + r0);
-            normals_of_block(p.seed, i0 >> 2, z);
-            // token tiles never straddle pair_rows (checked on the host)
-            se = (p.pair_rows > 0 && w.tok0 >= p.pair_rows) ? -p.sign_eps : p.sign_eps;
+          float z[kScaleRows][4];
+          uint2 raw[kScaleRows];
+#pragma unroll
+          for (int j = 0; j < kScaleRows; ++j) {
+            z[j][0] = z[j][1] = z[j][2] = z[j][3] = 0.0f;
+            raw[j] = make_uint2(0u, 0u);
+            if (live && j < rows) {
+              if (p.sign_eps != 0.0f) {
+                const uint64_t i0 = L.idx_base + (uint64_t)(row0 + j) * (uint64_t)L.N + (uint64_t)(w.n0 + r0);
+                normals_of_block(p.seed, i0 >> 2, z[j]);
+              }
+              if (!Plan::kRawViaCopy) raw[j] = *reinterpret_cast<const uint2*>(L.scales + (size_t)(row0 + j) * L.N + w.n0 + r0);
+            }
           }
           uint8_t* const slot_mem = smem + Plan::kOffA + slot * Plan::kNibBytes;
-          uint2 raw = make_uint2(0u, 0u);
-          if (!Plan::kRawViaCopy && live) raw = *reinterpret_cast<const uint2*>(L.scales + (size_t)g * L.N + w.n0 + r0);
           // kRawViaCopy: the stored scales came with the nibbles' copy; their arrival also says that the slot was
           // free.  Otherwise: the slot is free once the de-quantisers have read its previous group.
           const bool got = Plan::kRawViaCopy ? mbar_wait_relaxed(bar_nib_raw(slot), gph, abort_flag)
                                              : mbar_wait_relaxed(bar_nib_free(slot), gph ^ 1u, abort_flag);
           if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
-          float sv[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-          if (live) {
-            if (Plan::kRawViaCopy)
-              raw = *reinterpret_cast<const uint2*>(slot_mem + 2 * kPackedTileBytes + kCookedScaleBytes + r0 * 2);
-            const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
-            const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
-            sv[0] = fmaf(se, z[0], __low2float(a)); sv[1] = fmaf(se, z[1], __high2float(a));
-            sv[2] = fmaf(se, z[2], __low2float(b)); sv[3] = fmaf(se, z[3], __high2float(b));
-          }
-          uint32_t cooked[8];
 #pragma unroll
-          for (int l = 0; l < 4; ++l) {
-            const __nv_bfloat16 hi = __float2bfloat16_rn(sv[l]);
-            const __nv_bfloat16 lo = __float2bfloat16_rn(sv[l] - __bfloat162float(hi));
-            const uint32_t h16 = (uint32_t)__bfloat16_as_ushort(hi), l16 = (uint32_t)__bfloat16_as_ushort(lo);
-            cooked[2 * l] = h16 | (h16 << 16);
-            cooked[2 * l + 1] = l16 | (l16 << 16);
+          for (int j = 0; j < kScaleRows; ++j) {
+            float sv[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+            if (live && j < rows) {
+              if (Plan::kRawViaCopy)
+                raw[j] = *reinterpret_cast<const uint2*>(slot_mem + Plan::kOffRawInSlot + j * kRawScaleBytes + r0 * 2);
+              const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&raw[j].x);
+              const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(&raw[j].y);
+              sv[0] = fmaf(se, z[j][0], __low2float(a)); sv[1] = fmaf(se, z[j][1], __high2float(a));
+              sv[2] = fmaf(se, z[j][2], __low2float(b)); sv[3] = fmaf(se, z[j][3], __high2float(b));
+            }
+            uint32_t cooked[8];
+#pragma unroll
+            for (int l = 0; l < 4; ++l) {
+              const __nv_bfloat16 hi = __float2bfloat16_rn(sv[l]);
+              const __nv_bfloat16 lo = __float2bfloat16_rn(sv[l] - __bfloat162float(hi));
+              const uint32_t h16 = (uint32_t)__bfloat16_as_ushort(hi), l16 = (uint32_t)__bfloat16_as_ushort(lo);
+              cooked[2 * l] = h16 | (h16 << 16);
+              cooked[2 * l + 1] = l16 | (l16 << 16);
+            }
+            uint4* dst = reinterpret_cast<uint4*>(slot_mem + Plan::kOffCookedInSlot + j * kCookedScaleBytes + r0 * 8);
+            dst[0] = make_uint4(cooked[0], cooked[1], cooked[2], cooked[3]);
+            dst[1] = make_uint4(cooked[4], cooked[5], cooked[6], cooked[7]);
           }
-          uint4* dst = reinterpret_cast<uint4*>(slot_mem + 2 * kPackedTileBytes + r0 * 8);
-          dst[0] = make_uint4(cooked[0], cooked[1], cooked[2], cooked[3]);
-          dst[1] = make_uint4(cooked[4], cooked[5], cooked[6], cooked[7]);
           __syncwarp();
           if (lane == 0) mbar_arrive(bar_nib_full(slot));
         }
@@ -696,15 +736,28 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
       __nv_bfloat162 s_hi, s_lo;
       *reinterpret_cast<uint32_t*>(&s_hi) = 0u;
       *reinterpret_cast<uint32_t*>(&s_lo) = 0u;
-      // nibbles of one 16-byte unit (32 consecutive k of this thread's row) -> 16 x bf16x2 (u - 8) * s'
+      // table mode: this lane's copy of the codebook (entry e at + 128 e)
+      const uint32_t lut_lane = base + Plan::kOffLut + (uint32_t)lane * 4u;
+      // nibbles of one 16-byte unit (32 consecutive k of this thread's row) -> 16 x bf16x2 (u - 8) * s', or
+      // table[u] * s' in table mode
       auto dequant16 = [&](const uint4& pk, uint32_t (&outw)[16]) {
         const uint32_t words[4] = {pk.x, pk.y, pk.z, pk.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
 #pragma unroll
           for (int pp = 0; pp < 4; ++pp) {
-            uint32_t x = ((words[i] >> (4 * pp)) & 0x000F000Fu) | 0x43004300u;     // bf16x2 {128 + u_lo, 128 + u_hi}
-            __nv_bfloat162 q2 = __hsub2(*reinterpret_cast<__nv_bfloat162*>(&x), magic_bias);   // exact u - 8
+            __nv_bfloat162 q2;
+            if (LUT) {
+              const uint32_t x = (words[i] >> (4 * pp)) & 0x000F000Fu;             // codes of k = 2 j (low half) and 2 j + 1
+              uint32_t ta, tb;
+              asm volatile("ld.shared.b32 %0, [%1];" : "=r"(ta) : "r"(lut_lane + ((x & 0xFu) << 7)));
+              asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tb) : "r"(lut_lane + (x >> 9)));      // (x >> 16) * 128
+              const uint32_t t2 = (ta & 0x0000FFFFu) | (tb & 0xFFFF0000u);
+              q2 = *reinterpret_cast<const __nv_bfloat162*>(&t2);
+            } else {
+              uint32_t x = ((words[i] >> (4 * pp)) & 0x000F000Fu) | 0x43004300u;   // bf16x2 {128 + u_lo, 128 + u_hi}
+              q2 = __hsub2(*reinterpret_cast<__nv_bfloat162*>(&x), magic_bias);     // exact u - 8
+            }
             __nv_bfloat162 w2 = __hfma2(q2, s_hi, __hmul2(q2, s_lo));
             outw[i * 4 + pp] = *reinterpret_cast<uint32_t*>(&w2);                  // k = 32 h + 2 j, 2 j + 1 in register j
           }
@@ -725,11 +778,11 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
           // the nibble slot is full: nibbles landed, perturbed scales written
           if (!__all_sync(0xffffffffu, mbar_wait(bar_nib_full(nslot), nph, abort_flag))) { ok = false; break; }
           const uint8_t* const slot_mem = smem + Plan::kOffA + nslot * Plan::kNibBytes;
-          {
-            const uint2 c = *reinterpret_cast<const uint2*>(slot_mem + 2 * kPackedTileBytes + r * 8);
-            *reinterpret_cast<uint32_t*>(&s_hi) = c.x;
-            *reinterpret_cast<uint32_t*>(&s_lo) = c.y;
-          }
+          // perturbed scale of this row: one per group (int4) or one per k-block (table mode)
+          uint2 cs[kScaleRows];
+#pragma unroll
+          for (int j = 0; j < kScaleRows; ++j)
+            cs[j] = *reinterpret_cast<const uint2*>(slot_mem + Plan::kOffCookedInSlot + j * kCookedScaleBytes + r * 8);
           // this row's 64 k of each k-block: two 16-byte units (32 k each)
           const uint8_t* src = slot_mem + r * 16;
           uint4 pk[4];
@@ -750,6 +803,11 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4) {
             if (q4 < 2 || two) {
+              if ((q4 & 1) == 0) {
+                const uint2 c = cs[LUT ? (q4 >> 1) : 0];
+                *reinterpret_cast<uint32_t*>(&s_hi) = c.x;
+                *reinterpret_cast<uint32_t*>(&s_lo) = c.y;
+              }
               dequant16(pk[q4], outw);
               tmem_st16(a_lane_base + (uint32_t)((slot * 2 + (q4 >> 1)) * kATmemColsPerStage + (q4 & 1) * 16), outw);
             }
@@ -989,11 +1047,11 @@ int sm_count() {
   return n;
 }
 
-template <int TOK, bool DEQUANT, int OUT_MODE>
+template <int TOK, int WMODE, int OUT_MODE>
 int launch_one(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorMap* ty, const GemmParams& p,
                cudaStream_t st) {
-  using Plan = SmemPlan<TOK, DEQUANT, OUT_MODE>;
-  auto kern = w4a16_gemm_kernel<TOK, DEQUANT, OUT_MODE>;
+  using Plan = SmemPlan<TOK, WMODE, OUT_MODE>;
+  auto kern = w4a16_gemm_kernel<TOK, WMODE, OUT_MODE>;
   static std::atomic<unsigned long long> configured{0};      // per instantiation, one bit per device
   if (first_use_on_device(configured))
     QZO_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Plan::kDynamicBytes));
@@ -1002,15 +1060,15 @@ int launch_one(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorMap* 
   return QZO_OK;
 }
 
-template <bool DEQUANT, int OUT_MODE>
+template <int WMODE, int OUT_MODE>
 int launch_tok(int tok, const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorMap* ty, const GemmParams& p,
                cudaStream_t st) {
   switch (tok) {
-    case 16: return launch_one<16, DEQUANT, OUT_MODE>(tx, tw, ty, p, st);
-    case 32: return launch_one<32, DEQUANT, OUT_MODE>(tx, tw, ty, p, st);
-    case 64: return launch_one<64, DEQUANT, OUT_MODE>(tx, tw, ty, p, st);
-    case 128: return launch_one<128, DEQUANT, OUT_MODE>(tx, tw, ty, p, st);
-    default: return launch_one<256, DEQUANT, OUT_MODE>(tx, tw, ty, p, st);
+    case 16: return launch_one<16, WMODE, OUT_MODE>(tx, tw, ty, p, st);
+    case 32: return launch_one<32, WMODE, OUT_MODE>(tx, tw, ty, p, st);
+    case 64: return launch_one<64, WMODE, OUT_MODE>(tx, tw, ty, p, st);
+    case 128: return launch_one<128, WMODE, OUT_MODE>(tx, tw, ty, p, st);
+    default: return launch_one<256, WMODE, OUT_MODE>(tx, tw, ty, p, st);
   }
 }
 
@@ -1059,9 +1117,11 @@ size_t gemm_workspace_bytes(int M, int K, int N) {
 // from int4 and perturbed scales.
 // pair_rows > 0: rows [0, pair_rows) are perturbed with sign * eps, rows [pair_rows, M) with -sign * eps;
 // pair_rows must be a multiple of the token tile of M (see paired_rows_ok).
+// lut16 (host, 16 floats) non-null: table mode: the nibbles index that table and the scales are [ceil(K/64)][N], one
+// row per block of 64 k; null: int4 with one row of scales per group of 128 k.
 int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const GemmLinear* lins, int n_lin,
                                 uint64_t seed, int sign, float eps, int pair_rows, void* d_ws, size_t ws_bytes,
-                                int* d_status, cudaStream_t st) {
+                                int* d_status, cudaStream_t st, const float* lut16) {
   if (M <= 0 || K <= 0 || (K % 8) != 0 || n_lin < 1 || n_lin > kMaxGroupedLinears) return QZO_ERR_BAD_ARG;
   if (pair_rows != 0 && !paired_rows_ok(M, pair_rows)) return QZO_ERR_BAD_ARG;
   for (int j = 0; j < n_lin; ++j)
@@ -1075,7 +1135,7 @@ int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const Ge
     if (any_split) {
       for (int j = 0; j < n_lin; ++j)
         QZO_TRY(launch_perturbed_gemm_group(d_x, M, K, lins + j, 1, seed, sign, eps, pair_rows, d_ws, ws_bytes, d_status,
-                                            st));
+                                            st, lut16));
       return QZO_OK;
     }
   }
@@ -1090,6 +1150,7 @@ int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const Ge
   p.sign_eps = (float)sign * eps;
   p.pair_rows = pair_rows;
   p.status = d_status;
+  if (lut16) memcpy(p.lut, lut16, sizeof(p.lut));
   const int splits = (n_lin == 1) ? gemm_splits(M, K, lins[0].N) : 1;
   for (int j = 0; j < n_lin; ++j) {
     LinearDesc& L = p.lin[j];
@@ -1111,7 +1172,7 @@ int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const Ge
     p.splits = 1;
     p.kb_per_split = ceil_div(p.num_kb, 2) * 2;
     p.total_units = p.tiles_n_total * p.m_tiles;
-    return launch_tok<true, kOutBf16>(tok, tx, tx, ty, p, st);
+    return lut16 ? launch_tok<kWTable16, kOutBf16>(tok, tx, tx, ty, p, st) : launch_tok<kWInt4, kOutBf16>(tok, tx, tx, ty, p, st);
   }
   const GemmLinear& g = lins[0];
   const int groups = ceil_div(K, kGroup);
@@ -1124,7 +1185,8 @@ int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const Ge
   p.kb_per_split = groups_per * 2;
   p.total_units = p.tiles_n_total * p.m_tiles * zdim;
   ty[0] = ty[1] = ty[2] = tx;                              // unused by the fp32 epilogue
-  QZO_TRY((launch_tok<true, kOutF32>(tok, tx, tx, ty, p, st)));
+  if (lut16) QZO_TRY((launch_tok<kWTable16, kOutF32>(tok, tx, tx, ty, p, st)));
+  else QZO_TRY((launch_tok<kWInt4, kOutF32>(tok, tx, tx, ty, p, st)));
   const int64_t total = (int64_t)M * g.N;
   QZO_LAUNCH(splitk_reduce_kernel, dim3((unsigned)ceil_div64(total, 256)), dim3(256), 0, st,
              reinterpret_cast<const float*>(d_ws), zdim, M, g.N, g.bias, g.out, g.ldo);
@@ -1151,7 +1213,7 @@ int launch_bf16_gemm_f32out(const __nv_bfloat16* d_x, const __nv_bfloat16* d_w, 
   p.m_tiles = ceil_div(M, tok);
   p.total_units = p.tiles_n_total * p.m_tiles;
   p.status = d_status;
-  return launch_tok<false, kOutF32>(tok, tx, tw, ty, p, st);
+  return launch_tok<kWBf16, kOutF32>(tok, tx, tw, ty, p, st);
 }
 
 }  // namespace qzo

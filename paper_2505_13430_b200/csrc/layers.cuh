@@ -44,9 +44,10 @@ struct GemmLinear {
 // pair_rows > 0: rows [0, pair_rows) take sign * eps, rows [pair_rows, M) take -sign * eps, so that one
 // launch serves both passes of a step; allowed when paired_rows_ok(M, pair_rows).
 bool paired_rows_ok(int M, int pair_rows);
+// lut16 (host pointer to 16 floats, or null): table mode, see gemm_w4a16.cu
 int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const GemmLinear* lins, int n_lin,
                                 uint64_t seed, int sign, float eps, int pair_rows, void* d_ws, size_t ws_bytes,
-                                int* d_status, cudaStream_t st);
+                                int* d_status, cudaStream_t st, const float* lut16 = nullptr);
 int launch_bf16_gemm_f32out(const __nv_bfloat16* d_x, const __nv_bfloat16* d_w, float* d_out, int M, int K, int N,
                             int* d_status, cudaStream_t st);
 }  // namespace qzo

@@ -37,14 +37,14 @@ def gemm_bytes(M, K, N):
     return K * N // 2 + 2 * ((K + 127) // 128) * N + 2 * M * K + 2 * M * N
 
 
-def run_shape(M, K, N, iters, sign=1, reps=9, settle=1.0, pass_ms=4.0):
+def run_shape(M, K, N, iters, sign=1, reps=9, settle=1.0, pass_ms=4.0, table16=False):
     per_set = gemm_bytes(M, K, N)
     n_sets = max(2, min(64, (2 * L2_BYTES) // per_set + 1))
     sets = []
     for i in range(n_sets):
         x = torch.randn((M, K), device="cuda", dtype=torch.float32).bfloat16()
         words = torch.randint(-2 ** 31, 2 ** 31 - 1, (K // 8, N), device="cuda", dtype=torch.int32)
-        s = (torch.rand(((K + 127) // 128, N), device="cuda") * 0.015 + 0.005).bfloat16()
+        s = (torch.rand(((K + 63) // 64 if table16 else (K + 127) // 128, N), device="cuda") * 0.015 + 0.005).bfloat16()
         wq = qzo.qzo_repack_int4(words, K, N)
         y = torch.empty((M, N), device="cuda", dtype=torch.bfloat16)
         sets.append((x, wq, s, y))
@@ -54,9 +54,14 @@ def run_shape(M, K, N, iters, sign=1, reps=9, settle=1.0, pass_ms=4.0):
     ws = torch.empty((max(need, 256),), dtype=torch.uint8, device="cuda")
     status = torch.zeros((1,), dtype=torch.int32, device="cuda")
 
+    table = [(-1.0 + 2.0 * i / 15.0) ** 3 for i in range(16)]        # any 16 values: the kernel looks them up
+
     def call(i):
         x, wq, s, y = sets[i % n_sets]
-        qzo.qzo_perturbed_gemm(x, wq, s, M, K, N, 42, 0, sign, 1e-3, y=y, workspace=ws, status=status)
+        if table16:
+            qzo.qzo_perturbed_gemm_table16(x, wq, s, table, M, K, N, 42, 0, sign, 1e-3, y=y, workspace=ws, status=status)
+        else:
+            qzo.qzo_perturbed_gemm(x, wq, s, M, K, N, 42, 0, sign, 1e-3, y=y, workspace=ws, status=status)
 
     for i in range(max(3, n_sets)):
         call(i)
@@ -105,13 +110,15 @@ def main():
     ap.add_argument("--iters", type=int, default=50)
     ap.add_argument("--settle", type=float, default=1.0, help="idle seconds before each shape is timed")
     ap.add_argument("--json", action="store_true")
+    ap.add_argument("--table16", action="store_true",
+                    help="time the 16-entry-codebook / block-64 prologue (NF4-style storage) instead of int4 / group 128")
     args = ap.parse_args()
     bw, tf, src = peaks()
     rows = []
     for shape in args.shapes.split(","):
         K, N = (int(v) for v in shape.split("x"))
         for M in (int(v) for v in args.tokens.split(",")):
-            us, best_us, n_sets = run_shape(M, K, N, args.iters, settle=args.settle)
+            us, best_us, n_sets = run_shape(M, K, N, args.iters, settle=args.settle, table16=args.table16)
             t_hbm = gemm_bytes(M, K, N) / (bw * 1e9) * 1e6
             t_mma = 2.0 * M * K * N / (tf * 1e12) * 1e6
             roof = max(t_hbm, t_mma)

@@ -28,7 +28,7 @@ EXPORTS = (
     "qzo_update_scales", "qzo_step", "qzo_step_host", "qzo_debug_set_capture", "qzo_debug_layer_output",
     "qzo_device_status", "qzo_launch_count", "qzo_profile_gemms", "qzo_profile_read",
     "qzo_step_begin", "qzo_step_finish", "qzo_get_scales", "qzo_set_scales", "qzo_debug_set_status",
-    "qzo_joint_workspace_bytes", "qzo_enable_joint_spsa",
+    "qzo_joint_workspace_bytes", "qzo_enable_joint_spsa", "qzo_perturbed_gemm_table16",
 )
 
 
@@ -74,6 +74,7 @@ def _load():
         "qzo_unpack_kernel_layout": (ci, [vp, ci, ci, vp, vp]),
         "qzo_gemm_workspace_bytes": (ci, [ci, ci, ci, P(sz)]),
         "qzo_perturbed_gemm": (ci, [vp, vp, vp, vp, vp, ci, ci, ci, u64, u64, ci, cf, vp, sz, vp, vp]),
+        "qzo_perturbed_gemm_table16": (ci, [vp, vp, vp, P(cf), vp, vp, ci, ci, ci, u64, u64, ci, cf, vp, sz, vp, vp]),
         "qzo_perturbed_gemm_noalloc": (ci, [vp, vp, vp, vp, vp, ci, ci, ci, u64, u64, ci, cf, vp, vp]),
         "qzo_update_scales_flat": (ci, [vp, i64, u64, u64, cf, cf, cf, vp]),
         "qzo_num_scales": (ci, [P(ModelDesc), P(i64), P(i64)]),
@@ -203,6 +204,25 @@ def qzo_perturbed_gemm(x, wq, scales, M, K, N, seed, scale_index_base, sign, eps
     _check(_lib.qzo_perturbed_gemm(_ptr(x), _ptr(wq), _ptr(scales), _ptr(bias), _ptr(y), M, K, N, seed,
                                    scale_index_base, sign, eps, _ptr(workspace), ws_bytes, _ptr(status), _stream()),
            "qzo_perturbed_gemm")
+    return y
+
+
+def qzo_perturbed_gemm_table16(x, codes_wq, scales, table16, M, K, N, seed, scale_index_base, sign, eps, bias=None, y=None,
+                               workspace=None, status=None):
+    """Y = X W' for 4-bit codes into a 16-entry table with one bf16 scale per block of 64 rows (NF4-style storage);
+    codes_wq is qzo_repack_int4 of the codes packed like int4 nibbles; table16: 16 floats (any sequence)."""
+    _cuda(x, torch.bfloat16), _cuda(codes_wq, torch.uint8), _cuda(scales, torch.bfloat16)
+    assert scales.shape[0] == (K + 63) // 64
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.bfloat16, device=x.device)
+    need = qzo_gemm_workspace_bytes(M, K, N)
+    if workspace is None and need:
+        workspace = torch.empty((need,), dtype=torch.uint8, device=x.device)
+    ws_bytes = workspace.numel() if workspace is not None else 0
+    table = (ctypes.c_float * 16)(*[float(v) for v in table16])
+    _check(_lib.qzo_perturbed_gemm_table16(_ptr(x), _ptr(codes_wq), _ptr(scales), table, _ptr(bias), _ptr(y), M, K, N, seed,
+                                           scale_index_base, sign, eps, _ptr(workspace), ws_bytes, _ptr(status), _stream()),
+           "qzo_perturbed_gemm_table16")
     return y
 
 
