@@ -278,6 +278,16 @@ int qzo_debug_set_capture(qzo_model* m, int layer);
  * (rows of the sign +1 copy first).  bytes below the size needed: QZO_ERR_BAD_ARG. */
 int qzo_debug_layer_output(qzo_model* m, int layer, int which, void* d_out, size_t bytes);
 
+/* Test entry for the bounded device-side waits (failure detection without a fault): runs the perturbed GEMM
+ * (seed 1, sign +1, eps 1e-3, no bias, a problem without split-K) with the copies of quantisation group
+ * `skip_group` of every CTA announced but never issued and with every wait bounded by wait_limit_cycles
+ * (capped at the normal limit of about two seconds).  Every role of the kernel then runs out of its wait,
+ * the CTA drains the copies it did issue, frees its tensor memory and RETURNS; *d_status becomes non-zero.
+ * Nothing traps and nothing spins without bound.  The output is unspecified.  Later calls are unaffected. */
+int qzo_debug_gemm_wait_expiry(const void* d_x_bf16, const void* d_wq, const void* d_scales_bf16, void* d_y_bf16,
+                               int M, int K, int N, int skip_group, int64_t wait_limit_cycles, int* d_status,
+                               void* stream);
+
 /* Reads the device status word: bit 0 = a bounded device-side wait expired in some launch since init
  * (returns QZO_ERR_DEVICE_TIMEOUT), bit 1 = a token id outside [0, vocab) was seen (QZO_ERR_BAD_ARG);
  * 0 = nothing to report.  Synchronises. */

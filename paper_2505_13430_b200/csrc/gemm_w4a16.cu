@@ -96,6 +96,8 @@ struct GemmParams {
   float sign_eps;                 // sign * eps (0 when unperturbed)
   int pair_rows;                  // > 0: token rows from this one on take -sign_eps (both passes of a step in one launch)
   int* status;
+  long long wait_limit;           // cycles after which a device-side wait gives up
+  int skip_group;                 // >= 0 (tests only): the A producer announces this group's copies but does not issue them
   float lut[16];                  // table mode: the 16 codebook values (a nibble is an index into them)
 };
 
@@ -146,18 +148,18 @@ __device__ __forceinline__ bool mbar_poll(uint32_t bar, uint32_t parity) {
   return done != 0;
 }
 // Bounded wait: false when the limit expired or another thread of the CTA already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long limit) {
   if (mbar_poll(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
     if (mbar_poll(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitLimitCycles) return false;
+    if (clock64() - t0 > limit) return false;
   }
 }
 // Same bound, for waits that are long and not latency-critical: sleeps between polls so that the
 // waiting warp leaves the issue slots to the working ones.
-__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long limit) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t i = 1;; ++i) {
@@ -165,7 +167,7 @@ __device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity,
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 0x3F) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitLimitCycles) return false;
+      if (clock64() - t0 > limit) return false;
     }
   }
 }
@@ -435,6 +437,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  const long long wait_limit = p.wait_limit;      // bound of every wait, in cycles (about two seconds outside tests)
 
   const uint32_t bar0 = base + Plan::kOffBars;
   auto bar_b_full = [&](int s) { return bar0 + 8u * s; };                        // activation tile landed
@@ -520,7 +523,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         if (is_b) {
           for (int it = 0; it < w.nkb; it += kBGroup) {
             const int nk = min(kBGroup, w.nkb - it);          // k-blocks of this slot
-            if (!mbar_wait(bar_b_empty(ring.s), ring.ph ^ 1u, abort_flag)) { ok = false; break; }
+            if (!mbar_wait(bar_b_empty(ring.s), ring.ph ^ 1u, abort_flag, wait_limit)) { ok = false; break; }
             mbar_arrive_expect_tx(bar_b_full(ring.s), (uint32_t)(nk * Plan::kXTileBytes));
             for (int j = 0; j < nk; ++j)
               tma_load_2d(base + Plan::kOffB + (ring.s * kBGroup + j) * Plan::kXTileBytes, &tmap_x, bar_b_full(ring.s),
@@ -532,12 +535,16 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
           for (int it = 0; it < w.nkb; it += kAGroup) {
             const int kb = w.kb_begin + it;
             const int nk = min(kAGroup, w.nkb - it);         // k-blocks of this slot (the last group of an odd K has one)
-            if (!mbar_wait(bar_nib_free(ring.s), ring.ph ^ 1u, abort_flag)) { ok = false; break; }
+            if (!mbar_wait(bar_nib_free(ring.s), ring.ph ^ 1u, abort_flag, wait_limit)) { ok = false; break; }
             const uint32_t dst = base + Plan::kOffA + ring.s * Plan::kNibBytes;
             if (DEQUANT) {
+              // tests of the bounded waits: one group's copies are announced and never issued, so every wait
+              // that depends on them runs out
+              const bool skip = issued == p.skip_group;
               mbar_arrive_expect_tx(bar_nib_full(ring.s), (uint32_t)(nk * kPackedTileBytes));
-              bulk_load(dst, L.wq + ((size_t)(w.n0 / kTileN) * p.num_kb + kb) * kPackedTileBytes,
-                        (uint32_t)(nk * kPackedTileBytes), bar_nib_full(ring.s));
+              if (!skip)
+                bulk_load(dst, L.wq + ((size_t)(w.n0 / kTileN) * p.num_kb + kb) * kPackedTileBytes,
+                          (uint32_t)(nk * kPackedTileBytes), bar_nib_full(ring.s));
               // the group's stored scales of this tile's features travel with the nibbles (N is a multiple of 8
               // and the scale rows are 16-byte aligned, so is every run of them)
               if (Plan::kRawViaCopy) {
@@ -546,7 +553,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 const int rows = LUT ? nk : 1;
                 const int row0 = LUT ? kb : (kb >> 1);
                 mbar_arrive_expect_tx(bar_nib_raw(ring.s), raw_bytes * (uint32_t)rows);
-                for (int j = 0; j < rows; ++j)
+                for (int j = 0; j < rows && !skip; ++j)
                   bulk_load(dst + Plan::kOffRawInSlot + j * kRawScaleBytes, L.scales + (size_t)(row0 + j) * L.N + w.n0, raw_bytes,
                             bar_nib_raw(ring.s));
               }
@@ -569,7 +576,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
           // are waited for through the stored scales' barrier (issued last) where there is one
           const uint32_t bar = (is_b || !DEQUANT) ? bar_b_full(idx % stages)
                                                   : (Plan::kRawViaCopy ? bar_nib_raw(idx % stages) : bar_nib_full(idx % stages));
-          mbar_wait(bar, (uint32_t)(idx / stages) & 1u, never_set);
+          mbar_wait(bar, (uint32_t)(idx / stages) & 1u, never_set, wait_limit);
         }
         // a nibble copy issued just before an awaited scale copy may land a moment after it
         if (!is_b && Plan::kRawViaCopy) __nanosleep(50000);
@@ -596,7 +603,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             const long long t0 = clock64();
             do {
               seen = ld_acquire_shared(ready_addr);
-            } while (seen >= 0 && seen <= itg && clock64() - t0 < kWaitLimitCycles);
+            } while (seen >= 0 && seen <= itg && clock64() - t0 < wait_limit);
           }
           if (seen <= itg) { ok = false; break; }             // the watch warp gave up (-1), or the limit expired
         }
@@ -639,9 +646,9 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         const int j = it % kAGroup;
         bool got = true;
         // the epilogue warps must have drained the previous unit's accumulator
-        if (it == 0) got = mbar_wait(bar_acc_empty, ((uint32_t)useq & 1u) ^ 1u, abort_flag);
-        if (DEQUANT && j == 0) got = got && mbar_wait(bar_a_deq(ra.s), ra.ph, abort_flag);
-        if (it % kBGroup == 0) got = got && mbar_wait(bar_b_full(rb.s), rb.ph, abort_flag);
+        if (it == 0) got = mbar_wait(bar_acc_empty, ((uint32_t)useq & 1u) ^ 1u, abort_flag, wait_limit);
+        if (DEQUANT && j == 0) got = got && mbar_wait(bar_a_deq(ra.s), ra.ph, abort_flag, wait_limit);
+        if (it % kBGroup == 0) got = got && mbar_wait(bar_b_full(rb.s), rb.ph, abort_flag, wait_limit);
         __syncwarp();
         if (!got) {
           if (lane == 0) st_release_shared(ready_addr, -1);
@@ -693,8 +700,8 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
           uint8_t* const slot_mem = smem + Plan::kOffA + slot * Plan::kNibBytes;
           // kRawViaCopy: the stored scales came with the nibbles' copy; their arrival also says that the slot was
           // free.  Otherwise: the slot is free once the de-quantisers have read its previous group.
-          const bool got = Plan::kRawViaCopy ? mbar_wait_relaxed(bar_nib_raw(slot), gph, abort_flag)
-                                             : mbar_wait_relaxed(bar_nib_free(slot), gph ^ 1u, abort_flag);
+          const bool got = Plan::kRawViaCopy ? mbar_wait_relaxed(bar_nib_raw(slot), gph, abort_flag, wait_limit)
+                                             : mbar_wait_relaxed(bar_nib_free(slot), gph ^ 1u, abort_flag, wait_limit);
           if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
 #pragma unroll
           for (int j = 0; j < kScaleRows; ++j) {
@@ -776,7 +783,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
           const uint32_t gph = (uint32_t)(gig / kASlots) & 1u;
           const bool two = it + 1 < w.nkb;                    // the last group of an odd K has one k-block
           // the nibble slot is full: nibbles landed, perturbed scales written
-          if (!__all_sync(0xffffffffu, mbar_wait(bar_nib_full(nslot), nph, abort_flag))) { ok = false; break; }
+          if (!__all_sync(0xffffffffu, mbar_wait(bar_nib_full(nslot), nph, abort_flag, wait_limit))) { ok = false; break; }
           const uint8_t* const slot_mem = smem + Plan::kOffA + nslot * Plan::kNibBytes;
           // perturbed scale of this row: one per group (int4) or one per k-block (table mode)
           uint2 cs[kScaleRows];
@@ -797,7 +804,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
           __syncwarp();
           if (lane == 0) mbar_arrive(bar_nib_free(nslot));
           // the tensor-memory stages of the slot are free once the MMAs of their previous group retired
-          if (!__all_sync(0xffffffffu, mbar_wait(bar_a_empty(slot), gph ^ 1u, abort_flag))) { ok = false; break; }
+          if (!__all_sync(0xffffffffu, mbar_wait(bar_a_empty(slot), gph ^ 1u, abort_flag, wait_limit))) { ok = false; break; }
           tcgen05_fence_after();                              // orders the MMAs' reads of this slot before the stores below
           uint32_t outw[16];
 #pragma unroll
@@ -880,7 +887,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
       const LinearDesc& L = p.lin[w.lin];
       const int n = w.n0 + f;
       const float bias = (L.bias != nullptr && n < L.N && w.z == 0) ? L.bias[n] : 0.0f;
-      if (ew == 0 && !mbar_wait(bar_acc_full, (uint32_t)useq & 1u, abort_flag)) {
+      if (ew == 0 && !mbar_wait(bar_acc_full, (uint32_t)useq & 1u, abort_flag, wait_limit)) {
         *epi_stop = useq;
         __threadfence_block();
       }
@@ -1074,6 +1081,15 @@ int launch_tok(int tok, const CUtensorMap& tx, const CUtensorMap& tw, const CUte
 
 }  // namespace
 
+// Test hook of the bounded waits (see qzo_debug_gemm_wait_expiry): a shorter wait limit and a group whose copies
+// are withheld, for the launches of the calling thread while the hook is set.
+static thread_local long long g_debug_wait_limit = 0;
+static thread_local int g_debug_skip_group = -1;
+void set_gemm_wait_debug(long long limit_cycles, int skip_group) {
+  g_debug_wait_limit = limit_cycles > kWaitLimitCycles ? kWaitLimitCycles : limit_cycles;
+  g_debug_skip_group = skip_group;
+}
+
 // Split-K plan: number of K slices for a problem (1 = none).  Slices hold an even number of
 // k-blocks so that they start on a quantisation-group boundary.  The choice minimises a simple
 // cost model measured on B200: a unit costs a pipeline fill plus ~600 cycles per k-block whatever
@@ -1150,6 +1166,8 @@ int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const Ge
   p.sign_eps = (float)sign * eps;
   p.pair_rows = pair_rows;
   p.status = d_status;
+  p.wait_limit = g_debug_wait_limit > 0 ? g_debug_wait_limit : kWaitLimitCycles;
+  p.skip_group = g_debug_skip_group;
   if (lut16) memcpy(p.lut, lut16, sizeof(p.lut));
   const int splits = (n_lin == 1) ? gemm_splits(M, K, lins[0].N) : 1;
   for (int j = 0; j < n_lin; ++j) {
@@ -1213,6 +1231,8 @@ int launch_bf16_gemm_f32out(const __nv_bfloat16* d_x, const __nv_bfloat16* d_w, 
   p.m_tiles = ceil_div(M, tok);
   p.total_units = p.tiles_n_total * p.m_tiles;
   p.status = d_status;
+  p.wait_limit = kWaitLimitCycles;
+  p.skip_group = -1;
   return launch_tok<kWBf16, kOutF32>(tok, tx, tw, ty, p, st);
 }
 

@@ -48,6 +48,9 @@ bool paired_rows_ok(int M, int pair_rows);
 int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const GemmLinear* lins, int n_lin,
                                 uint64_t seed, int sign, float eps, int pair_rows, void* d_ws, size_t ws_bytes,
                                 int* d_status, cudaStream_t st, const float* lut16 = nullptr);
+// Test hook: later perturbed-GEMM launches of the calling thread use this wait limit (cycles; 0 = the normal
+// one) and withhold the copies of quantisation group `skip_group` of every CTA (-1 = none).
+void set_gemm_wait_debug(long long limit_cycles, int skip_group);
 int launch_bf16_gemm_f32out(const __nv_bfloat16* d_x, const __nv_bfloat16* d_w, float* d_out, int M, int K, int N,
                             int* d_status, cudaStream_t st);
 }  // namespace qzo

@@ -505,6 +505,16 @@ int qzo_perturbed_gemm_table16(const void* d_x_bf16, const void* d_codes, const 
                                      workspace_bytes, d_status, (cudaStream_t)stream, h_table16);
 }
 
+int qzo_debug_gemm_wait_expiry(const void* d_x_bf16, const void* d_wq, const void* d_scales_bf16, void* d_y_bf16, int M,
+                               int K, int N, int skip_group, int64_t wait_limit_cycles, int* d_status, void* stream) {
+  if (skip_group < 0 || wait_limit_cycles <= 0 || !d_status) return QZO_ERR_BAD_ARG;
+  set_gemm_wait_debug((long long)wait_limit_cycles, skip_group);
+  const int rc = qzo_perturbed_gemm(d_x_bf16, d_wq, d_scales_bf16, nullptr, d_y_bf16, M, K, N, 1, 0, +1, 1e-3f, nullptr, 0,
+                                    d_status, stream);
+  set_gemm_wait_debug(0, -1);
+  return rc;
+}
+
 int qzo_update_scales_flat(void* d_scales_bf16, int64_t count, uint64_t seed, uint64_t index_base, float lr, float g,
                            float clip, void* stream) {
   if (!d_scales_bf16 || count < 0 || (index_base % 4) || ((uintptr_t)d_scales_bf16 & 7) || !(clip >= 0.0f))

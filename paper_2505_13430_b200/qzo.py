@@ -28,7 +28,7 @@ EXPORTS = (
     "qzo_update_scales", "qzo_step", "qzo_step_host", "qzo_debug_set_capture", "qzo_debug_layer_output",
     "qzo_device_status", "qzo_launch_count", "qzo_profile_gemms", "qzo_profile_read",
     "qzo_step_begin", "qzo_step_finish", "qzo_get_scales", "qzo_set_scales", "qzo_debug_set_status",
-    "qzo_joint_workspace_bytes", "qzo_enable_joint_spsa", "qzo_perturbed_gemm_table16",
+    "qzo_joint_workspace_bytes", "qzo_enable_joint_spsa", "qzo_perturbed_gemm_table16", "qzo_debug_gemm_wait_expiry",
 )
 
 
@@ -75,6 +75,7 @@ def _load():
         "qzo_gemm_workspace_bytes": (ci, [ci, ci, ci, P(sz)]),
         "qzo_perturbed_gemm": (ci, [vp, vp, vp, vp, vp, ci, ci, ci, u64, u64, ci, cf, vp, sz, vp, vp]),
         "qzo_perturbed_gemm_table16": (ci, [vp, vp, vp, P(cf), vp, vp, ci, ci, ci, u64, u64, ci, cf, vp, sz, vp, vp]),
+        "qzo_debug_gemm_wait_expiry": (ci, [vp, vp, vp, vp, ci, ci, ci, ci, i64, vp, vp]),
         "qzo_perturbed_gemm_noalloc": (ci, [vp, vp, vp, vp, vp, ci, ci, ci, u64, u64, ci, cf, vp, vp]),
         "qzo_update_scales_flat": (ci, [vp, i64, u64, u64, cf, cf, cf, vp]),
         "qzo_num_scales": (ci, [P(ModelDesc), P(i64), P(i64)]),
@@ -224,6 +225,13 @@ def qzo_perturbed_gemm_table16(x, codes_wq, scales, table16, M, K, N, seed, scal
                                            scale_index_base, sign, eps, _ptr(workspace), ws_bytes, _ptr(status), _stream()),
            "qzo_perturbed_gemm_table16")
     return y
+
+
+def qzo_debug_gemm_wait_expiry(x, wq, scales, y, M, K, N, skip_group, wait_limit_cycles, status):
+    """Test entry: the GEMM with one group's copies withheld and a short wait limit; see include/qzo.h."""
+    _cuda(x, torch.bfloat16), _cuda(wq, torch.uint8), _cuda(scales, torch.bfloat16), _cuda(y, torch.bfloat16)
+    _check(_lib.qzo_debug_gemm_wait_expiry(_ptr(x), _ptr(wq), _ptr(scales), _ptr(y), M, K, N, skip_group, wait_limit_cycles,
+                                           _ptr(status), _stream()), "qzo_debug_gemm_wait_expiry")
 
 
 NOALLOC_SCRATCH_BYTES = 16 << 20
