@@ -1,11 +1,12 @@
 """One QZO step (oracle): Algorithm 1, Eq. 5 (Q-SPSA) and Eq. 6 (DDC).
 
-Two forms are given.  `step_literal` walks Algorithm 1 as printed: perturb the
-scales in place by +eps z, forward, by -2 eps z, forward, by +eps z (restore),
-then d, d' and the seeded update with max(., 0).  `step_functional` evaluates
-the same quantities from the untouched scales, Delta' = Delta + sign*eps*z,
-which is what the library does.  In exact arithmetic they agree; the tests
-require agreement to fp64 rounding.
+Two forms are given.  `step_literal` is the in-place form of Algorithm 1: the
+scales themselves are moved by +eps z before the first forward, by -2 eps z
+before the second and by +eps z afterwards (which restores them), then d, d'
+and the seeded update with max(., 0) follow.  `step_functional` evaluates the
+same quantities from the untouched scales, Delta' = Delta + sign*eps*z, which
+is what the library does.  In exact arithmetic they agree; the tests require
+agreement to fp64 rounding (the equivalence is the property being pinned).
 
 Storage rounding of the updated scale (bf16, ties to even) is a reading: the
 paper does not fix the dtype of Delta.  `lr * d'` is formed once in fp32 and
@@ -116,7 +117,7 @@ def _perturb_in_place(model, scale, seed):
 
 
 def step_literal(model, tokens, labels, seed, eps, lr, C):
-    """Algorithm 1 as printed, scales held in fp64 and mutated in place.
+    """Algorithm 1 in its in-place form, scales held in fp64 and mutated.
 
     Returns (l+, l-, d, d'); the model's scales end as fp64
     max(Delta_i - lr d' z_i, 0) without storage rounding.
