@@ -3,7 +3,8 @@
 * The standalone perturbed W4A16 GEMM on every K x N and token count of the sweep, in the launch
   configuration the sweep times (same entry point, same tile / split-K choice): sampled rows and
   columns (first and last tile, ragged edges, random ones) against the oracle, max relative 2e-2.
-* A full-width model truncated to two decoder blocks, at the benchmark's batch, through qzo_step (both
+* A full-width model truncated to four (Llama-2-7B shape) or two (OPT-6.7B shape) decoder blocks, at the
+  benchmark's batch, through qzo_step (both
   signs in one pass, the route the benchmark times): losses L+- within 1e-3 of the oracle's, the
   directional derivative printed beside the oracle's.
 * A Llama-2-7B-width block built for 4096 tokens and called with 16 and with 128 tokens (the split-K
@@ -116,11 +117,11 @@ def _oracle_and_gpu_model(lib, workload, n_layers, max_tokens):
     return cfg, om, gm
 
 
-@pytest.mark.parametrize("workload", ["llama7b", "opt6.7b"])
-def test_two_layer_full_width_step_losses_match_oracle(lib, workload):
+@pytest.mark.parametrize("workload,n_layers", [("llama7b", 4), ("opt6.7b", 2)])
+def test_truncated_full_width_step_losses_match_oracle(lib, workload, n_layers):
     c = inputs.CONFIGS[workload]
     B, S = c["batch"], c["seq"]
-    cfg, om, gm = _oracle_and_gpu_model(lib, workload, 2, B * S)
+    cfg, om, gm = _oracle_and_gpu_model(lib, workload, n_layers, B * S)
     tok, lab = inputs.tokens_and_labels(cfg, B, S, seed=7)
     seed, eps = 42, c["eps"]
     lp, lm, d, dc = gm.qzo_step(tok.cuda(), lab.cuda(), seed, eps, c["lr"], c["clip"])
@@ -128,7 +129,7 @@ def test_two_layer_full_width_step_losses_match_oracle(lib, workload):
     rp = omodel.forward_loss(om, tok.numpy(), lab.numpy(), seed, +1, eps)
     rm = omodel.forward_loss(om, tok.numpy(), lab.numpy(), seed, -1, eps)
     d_ref = (rp - rm) / (2 * eps)
-    print(f"{workload} x 2 layers, {B} x {S} tokens: L+ {lp:.6f} (oracle {rp:.6f})  L- {lm:.6f} (oracle {rm:.6f})  "
+    print(f"{workload} x {n_layers} layers, {B} x {S} tokens: L+ {lp:.6f} (oracle {rp:.6f})  L- {lm:.6f} (oracle {rm:.6f})  "
           f"d {d:.4f} (oracle {d_ref:.4f})")
     assert abs(lp - rp) <= 1e-3 and abs(lm - rm) <= 1e-3
     # d is a difference of two losses that agree to 1e-3 each: what that allows, and no more
@@ -158,4 +159,63 @@ def test_small_batch_on_a_model_planned_for_the_large_batch(lib, tokens):
     lp, lm, d, dc = gm.qzo_step(tok.cuda(), lab.cuda(), 5, 1e-3, 1e-5, 100.0)
     assert gm.qzo_device_status() == 0
     assert abs(lp - omodel.forward_loss(om, tok.numpy(), lab.numpy(), 5, +1, 1e-3)) <= tol_loss
+    gm.close()
+
+
+def test_table_mode_gemm_at_a_sweep_size_on_sampled_outputs(lib):
+    # the 16-entry-codebook / block-64 prologue at a full sweep shape, in the sweep's launch configuration
+    M, K, N = 1024, 4096, 11008
+    g = torch.Generator(device="cuda")
+    g.manual_seed(99)
+    x = torch.randn((M, K), generator=g, device="cuda", dtype=torch.float32).bfloat16()
+    words = torch.randint(-2 ** 31, 2 ** 31 - 1, (K // 8, N), generator=g, device="cuda", dtype=torch.int32)
+    s = (torch.rand(((K + 63) // 64, N), generator=g, device="cuda", dtype=torch.float32) * 0.03 + 0.01).bfloat16()
+    table = torch.sort(torch.rand((16,), generator=g, device="cuda") * 2 - 1).values.cpu().numpy()
+    wq = lib.qzo_repack_int4(words, K, N)
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    rng = np.random.default_rng(5)
+    rows = _sample(rng, M, [0, 255, 256, M - 1], 5)
+    cols = _sample(rng, N, [0, 127, 128, N - 1], 20)
+    codes = int4.unpack_int4(words[:, cols].cpu().numpy().view(np.uint32)).astype(np.int64) + 8
+    seed, base, eps = 31, 16, 1e-3
+    for sign in (+1, -1):
+        y = lib.qzo_perturbed_gemm_table16(x, wq, s, table.tolist(), M, K, N, seed, base, sign, eps, status=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        # the oracle on the sampled rows / columns: scales of the sampled columns with their logical indices
+        sp = s[:, cols].float().cpu().numpy().astype(np.float64)
+        idx = np.uint64(base) + np.arange(sp.shape[0], dtype=np.uint64)[:, None] * np.uint64(N) + np.asarray(cols, dtype=np.uint64)[None, :]
+        from oracle import philox
+        sp = sp + sign * eps * philox.normal_from_index(seed, idx).astype(np.float64)
+        w = sp[np.arange(K) // 64] * table.astype(np.float64)[codes]
+        ref = x[rows].float().cpu().numpy().astype(np.float64) @ w
+        got = y[rows][:, cols].float().cpu().numpy().astype(np.float64)
+        assert np.abs(got - ref).max() <= TOL * np.abs(ref).max(), sign
+
+
+def test_joint_mode_full_width_block_on_sampled_sequences(lib):
+    # joint SPSA at the Llama-2-7B width (one block, the benchmark's batch): block output, logits and loss
+    c = inputs.CONFIGS["llama7b"]
+    B, S = c["batch"], c["seq"]
+    cfg, om, gm = _oracle_and_gpu_model(lib, "llama7b", 1, B * S)
+    gm.qzo_enable_joint_spsa(1e-4)
+    tok, lab = inputs.tokens_and_labels(cfg, B, S, seed=7)
+    gm.qzo_debug_set_capture(0)
+    seed, eps = 42, c["eps"]
+    gm.qzo_forward_loss(tok.cuda(), lab.cuda(), seed, +1, eps)
+    hid = gm.qzo_debug_layer_output(0, 0, B * S).view(B, S, -1)
+    logits = gm.qzo_debug_layer_output(0, 1, B * S).view(B, S, -1)
+    for b in (0, B - 1):
+        cap = {}
+        omodel.forward_loss(om, tok[b:b + 1].numpy(), lab[b:b + 1].numpy(), seed, +1, eps, capture=cap, perturb_dense=True)
+        got_h = hid[b].float().cpu().numpy().astype(np.float64)
+        assert np.abs(got_h - cap["hidden"][0]).max() <= TOL * np.abs(cap["hidden"][0]).max(), b
+        got_l = logits[b].float().cpu().numpy().astype(np.float64)
+        assert np.abs(got_l - cap["logits"]).max() <= TOL * np.abs(cap["logits"]).max(), b
+    # whole step: both signs in one pass equal the single-sign calls bit for bit, also in joint mode
+    lp = gm.qzo_forward_loss(tok.cuda(), lab.cuda(), seed, +1, eps).cpu().clone()
+    lm = gm.qzo_forward_loss(tok.cuda(), lab.cuda(), seed, -1, eps).cpu().clone()
+    out = gm.qzo_step(tok.cuda(), lab.cuda(), seed, eps, c["lr"], 0.0)       # C = 0: nothing moves
+    assert np.float32(out[0]) == np.float32(lp[0]) and np.float32(out[1]) == np.float32(lm[0])
+    assert gm.qzo_device_status() == 0
     gm.close()
