@@ -185,7 +185,7 @@ int qzo_scale_layout(const qzo_model_desc* desc, int layer, int linear,
  * buffers hold 2 * max_tokens rows, because qzo_step runs both passes as one forward. */
 int qzo_workspace_bytes(const qzo_model_desc* desc, int max_tokens, size_t* bytes);
 
-/* Binds a model to caller-owned tensors (Algorithm 1 "Require": scales Delta, integer
+/* Binds a model to caller-owned tensors (the inputs of Algorithm 1: scales Delta, integer
  * weights theta_bar).  Tensors, by name:
  *   "embed" bf16 [V][d]; "lm_head" bf16 [V][d]; "pos_embed" bf16 [max_seq][d] (OPT);
  *   "final_norm_w" f32 [d] (+ "final_norm_b", OPT); "scales" bf16 [flat_entries] (trained in place);
@@ -200,7 +200,7 @@ int qzo_init_model(const qzo_model_desc* desc, const qzo_tensor* tensors, int n_
 int qzo_free_model(qzo_model* m);
 
 /* One forward pass, L(Delta' (.) theta_bar; B) with Delta' = Delta + sign eps z(seed)
- * (Algorithm 1, "1st/2nd forward pass"; sign 0 = unperturbed).  d_tokens, d_labels:
+ * (either forward pass of Algorithm 1; sign 0 = unperturbed).  d_tokens, d_labels:
  * int32 [B][S]; label -100 is ignored; loss = mean next-token cross entropy over kept
  * positions, written to d_loss (float, device). */
 int qzo_forward_loss(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S,
@@ -241,8 +241,9 @@ int qzo_step_begin(qzo_model* m, const int32_t* d_tokens, const int32_t* d_label
 int qzo_step_finish(qzo_model* m, const float* d_sums, uint64_t seed, float eps, float lr, float clip,
                     float* h_out);
 
-/* Joint mode (Sec. 3.2.1, closing remark: Q-SPSA on the scales combined with SPSA on the un-quantised
- * parts; Sec. 4.1: "the un-quantized parts are jointly fine-tuned using the regular SPSA and ZO-SGD").
+/* Joint mode (Sec. 3.2.1, closing remark: Q-SPSA on the scales may be combined with SPSA on the
+ * un-quantised parts; Sec. 4.1, implementation details: the experiments with codebook weights train the
+ * un-quantised parts that way, with plain SPSA and ZO-SGD).
  * After qzo_enable_joint_spsa every perturbed forward (sign +1 / -1) also perturbs the embedding matrix, the
  * lm_head matrix and every norm gain (and norm bias, OPT) as theta + sign eps z (Def. 3.1), and every step
  * also updates them in place, theta <- theta - lr_dense d' z (Def. 3.2; no clamp, that belongs to the
@@ -260,7 +261,7 @@ int qzo_enable_joint_spsa(qzo_model* m, void* d_workspace, size_t workspace_byte
 int qzo_step_host(qzo_model* m, const int32_t* h_tokens, const int32_t* h_labels, int B, int S,
                   uint64_t seed, float eps, float lr, float clip, float* h_out);
 
-/* The trainable state (Algorithm 1 "Require": the quantisation scales Delta that the caller hands over
+/* The trainable state (the inputs of Algorithm 1: the quantisation scales Delta that the caller hands over
  * and gets back).  linear_id = layer * L + position, L = 7 (Llama: q,k,v,o,gate,up,down) or 6 (OPT:
  * q,k,v,o,fc1,fc2): copies that linear's bf16 [G][N] scales out of / into the model's flat buffer;
  * linear_id = -1: the whole flat buffer (qzo_num_scales entries).  d_bf16 is a device pointer; `bytes` must

@@ -1,8 +1,8 @@
 """Philox4x32-10 counter RNG and the z(seed, index) map (oracle, fp64).
 
 The paper only says that a random seed is stored and the Gaussian direction z
-is regenerated from it when needed (Sec. 3.1, MeZO seed trick; Algorithm 1,
-"Reset random number generator with seed s").  The generator used here is the
+is regenerated from it when needed (Sec. 3.1, MeZO seed trick; Algorithm 1
+re-seeds its generator before every sweep over the scales).  The generator used here is the
 published Philox4x32-10 (Salmon et al., SC'11) keyed on the 64-bit seed, with
 the logical scale index as the counter, so that z_i is a pure function of
 (seed, i) and can be regenerated in any order.
