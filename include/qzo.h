@@ -86,7 +86,7 @@ int qzo_unpack_int4(const uint32_t* d_qpacked, int K, int N, int8_t* d_q, void* 
 /* Size in bytes of the kernel-layout copy of a K x N int4 weight. */
 int qzo_repacked_bytes(int K, int N, size_t* bytes);
 /* interchange -> kernel layout (done once; theta_bar is fixed for the whole run,
- * Algorithm 1 "quantized weights").  d_out: `bytes` from qzo_repacked_bytes, 256-aligned. */
+ * the integer weights that Algorithm 1 takes as an input).  d_out: `bytes` from qzo_repacked_bytes, 256-aligned. */
 int qzo_repack_int4(const uint32_t* d_qpacked, int K, int N, void* d_out, size_t out_bytes,
                     void* stream);
 /* kernel layout -> int8 q [K][N]: what the GEMM's prologue sees (bit-exact check). */
