@@ -1095,8 +1095,7 @@ void set_gemm_wait_debug(long long limit_cycles, int skip_group) {
 // cost model measured on B200: a unit costs a pipeline fill plus ~600 cycles per k-block whatever
 // the token tile, the units run in rounds of one per SM, and a split adds the fp32 partial sums'
 // round trip and a second launch.  Depends on the shape only, so results are reproducible.
-int gemm_splits(int M, int K, int N) {
-  const int tok = pick_tok_tile(M);
+static int gemm_splits_tok(int M, int K, int N, int tok) {
   if (tok > 128) return 1;                       // 256-token tiles: plenty of units, tensor-bound
   const int tiles = ceil_div(N, kTileN) * ceil_div(M, tok);
   const int groups = ceil_div(K, kGroup);
@@ -1117,14 +1116,25 @@ int gemm_splits(int M, int K, int N) {
   return best;
 }
 
-// Whether a launch over M token rows may switch the perturbation sign at row `pair_rows`: the
-// boundary must fall between two token tiles.
-bool paired_rows_ok(int M, int pair_rows) {
-  return pair_rows > 0 && pair_rows < M && pair_rows % pick_tok_tile(M) == 0;
+int gemm_splits(int M, int K, int N) { return gemm_splits_tok(M, K, N, pick_tok_tile(M)); }
+
+// Token tile of a launch over M rows.  A launch that switches the perturbation sign at row `pair_rows`
+// (M = 2 pair_rows) takes the tile of pair_rows rows and needs pair_rows to be a multiple of it, so that
+// the boundary falls between two token tiles and the launch has exactly the units of the two single-sign
+// launches it replaces: pair_rows in {16, 32, 64, 128} or a multiple of 256; 0 otherwise.
+static int launch_tok_tile(int M, int pair_rows) {
+  if (pair_rows <= 0) return pick_tok_tile(M);
+  const int t = pick_tok_tile(pair_rows);
+  return pair_rows % t == 0 ? t : 0;
 }
 
-size_t gemm_workspace_bytes(int M, int K, int N) {
-  const int splits = gemm_splits(M, K, N);
+bool paired_rows_ok(int M, int pair_rows) {
+  return pair_rows > 0 && pair_rows < M && launch_tok_tile(M, pair_rows) > 0;
+}
+
+size_t gemm_workspace_bytes(int M, int K, int N, int pair_rows) {
+  const int tok = launch_tok_tile(M, pair_rows);
+  const int splits = tok > 0 ? gemm_splits_tok(pair_rows > 0 ? pair_rows : M, K, N, tok) : 1;
   if (splits <= 1) return 0;
   return (size_t)splits * M * N * sizeof(float);
 }
@@ -1132,7 +1142,7 @@ size_t gemm_workspace_bytes(int M, int K, int N) {
 // Y_j = X W'_j (+ bias_j) for up to three linears that share X, with W'_j de-quantised
 // from int4 and perturbed scales.
 // pair_rows > 0: rows [0, pair_rows) are perturbed with sign * eps, rows [pair_rows, M) with -sign * eps;
-// pair_rows must be a multiple of the token tile of M (see paired_rows_ok).
+// see paired_rows_ok for the row counts that allow it.
 // lut16 (host, 16 floats) non-null: table mode: the nibbles index that table and the scales are [ceil(K/64)][N], one
 // row per block of 64 k; null: int4 with one row of scales per group of 128 k.
 int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const GemmLinear* lins, int n_lin,
@@ -1143,11 +1153,14 @@ int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const Ge
   for (int j = 0; j < n_lin; ++j)
     if (lins[j].N <= 0 || (lins[j].N % 8) != 0 || (lins[j].idx_base % 4) != 0 || (lins[j].ldo % 8) != 0)
       return QZO_ERR_BAD_ARG;
-  const int tok = pick_tok_tile(M);
+  const int tok = launch_tok_tile(M, pair_rows);
+  // A paired launch slices K like each of the two single-sign launches it replaces, so that both ways of
+  // running a step add up the same partial sums in the same order.
+  const int m_plan = pair_rows > 0 ? pair_rows : M;
   // split-K only pays for small token counts; grouped launches of such problems go one by one
   if (n_lin > 1) {
     bool any_split = false;
-    for (int j = 0; j < n_lin; ++j) any_split = any_split || gemm_splits(M, K, lins[j].N) > 1;
+    for (int j = 0; j < n_lin; ++j) any_split = any_split || gemm_splits_tok(m_plan, K, lins[j].N, tok) > 1;
     if (any_split) {
       for (int j = 0; j < n_lin; ++j)
         QZO_TRY(launch_perturbed_gemm_group(d_x, M, K, lins + j, 1, seed, sign, eps, pair_rows, d_ws, ws_bytes, d_status,
@@ -1169,7 +1182,7 @@ int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const Ge
   p.wait_limit = g_debug_wait_limit > 0 ? g_debug_wait_limit : kWaitLimitCycles;
   p.skip_group = g_debug_skip_group;
   if (lut16) memcpy(p.lut, lut16, sizeof(p.lut));
-  const int splits = (n_lin == 1) ? gemm_splits(M, K, lins[0].N) : 1;
+  const int splits = (n_lin == 1) ? gemm_splits_tok(m_plan, K, lins[0].N, tok) : 1;
   for (int j = 0; j < n_lin; ++j) {
     LinearDesc& L = p.lin[j];
     L.wq = reinterpret_cast<const uint8_t*>(lins[j].wq);

@@ -28,9 +28,10 @@ int launch_ddc(const float* sums4, float eps, float lr, float lr_dense, float cl
                cudaStream_t st);
 
 // gemm_w4a16.cu
-constexpr int kMaxSplitTokens = 128;   // launches with more tokens never split along K
+constexpr int kMaxSplitTokens = 128;   // token tiles above this never split along K
 int gemm_splits(int M, int K, int N);
-size_t gemm_workspace_bytes(int M, int K, int N);
+// pair_rows > 0: the launch switches the perturbation sign at that row (see paired_rows_ok)
+size_t gemm_workspace_bytes(int M, int K, int N, int pair_rows = 0);
 // One linear of a grouped launch: Y = X W' (+ bias), Y bf16 [M][ldo].
 constexpr int kMaxGroupedLinears = 3;
 struct GemmLinear {
@@ -42,7 +43,7 @@ struct GemmLinear {
   uint64_t idx_base;              // logical index of scale [0][0]
 };
 // pair_rows > 0: rows [0, pair_rows) take sign * eps, rows [pair_rows, M) take -sign * eps, so that one
-// launch serves both passes of a step; allowed when paired_rows_ok(M, pair_rows).
+// launch serves both passes of a step; allowed when paired_rows_ok(M, pair_rows): pair_rows in {16, 32, 64, 128} or a multiple of 256.
 bool paired_rows_ok(int M, int pair_rows);
 // lut16 (host pointer to 16 floats, or null): table mode, see gemm_w4a16.cu
 int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const GemmLinear* lins, int n_lin,

@@ -174,6 +174,8 @@ int plan_workspace(const qzo_model_desc& d, int max_tokens, WsPlan* p) {
   size_t gb = 0;
   for (int i = 0; i < nl; ++i) {
     for (int M = 1; M <= std::min(T, kMaxSplitTokens); ++M) gb = std::max(gb, gemm_workspace_bytes(M, ls[i].K, ls[i].N));
+    for (int half = 16; half <= std::min(max_tokens, kMaxSplitTokens); half *= 2)      // paired steps of few tokens
+      gb = std::max(gb, gemm_workspace_bytes(2 * half, ls[i].K, ls[i].N, half));
     gb = std::max(gb, std::max(gemm_workspace_bytes(T, ls[i].K, ls[i].N), gemm_workspace_bytes(max_tokens, ls[i].K, ls[i].N)));
   }
   p->gemm_bytes = gb;

@@ -193,15 +193,18 @@ def test_empty_and_minimal_calls(lib):
 
 @pytest.mark.parametrize("name", ["tiny", "tiny_opt"])
 def test_step_in_one_pass_equals_two_separate_passes(lib, name):
-    # With 256 tokens the step runs both perturbation signs as one forward over two copies of the
-    # batch; with 192 tokens (no token-tile boundary between the copies) it runs two forwards.  Either
-    # way the losses it reports are, bit for bit, those of the single-sign entry point, and they match
-    # the oracle.
+    # With 16, 32, 64, 128 tokens or a multiple of 256 the step runs both perturbation signs as one forward
+    # over two copies of the batch (the boundary between the copies falls between two token tiles); with
+    # any other count (192, 144, 8 here) it runs two forwards.  Either way the losses it reports are, bit
+    # for bit, those of the single-sign entry point, and they match the oracle.
     cfg, c, om, gm, tok, lab = _setup(lib, name)
     seed, eps = 17, c["eps"]
-    for rows in (c["batch"], c["batch"] - 1, 0):
-        # rows = 0 stands for one sequence of 8 tokens (the smallest token tile; a step of two passes)
-        t, l = (tok[:rows].contiguous(), lab[:rows].contiguous()) if rows else (tok[:1, :8].contiguous(), lab[:1, :8].contiguous())
+    cases = [(c["batch"], c["seq"]), (c["batch"] - 1, c["seq"]), (1, 8), (1, 16), (1, 32), (2, 32), (4, 32)]
+    if c["seq"] == 64:
+        cases.append((2, 64))
+    for nb, ns in cases:
+        t, l = tok[:nb, :ns].contiguous(), lab[:nb, :ns].contiguous()
+        rows = (nb, ns)
         t_d, l_d = t.cuda(), l.cuda()
         lp = gm.qzo_forward_loss(t_d, l_d, seed, +1, eps).cpu().clone()
         lm = gm.qzo_forward_loss(t_d, l_d, seed, -1, eps).cpu().clone()
