@@ -211,10 +211,13 @@ int qzo_forward_loss(qzo_model* m, const int32_t* d_tokens, const int32_t* d_lab
 int qzo_update_scales(qzo_model* m, uint64_t seed, float lr, float g, float clip);
 
 /* Whole step of Algorithm 1 on device-resident tokens: two forwards (sign +1, -1), d, d' and
- * the update, with d formed on the device.  When B*S is a multiple of the GEMM's token tile the
+ * the update, with d formed on the device.  When B*S is 16, 32, 64, 128 or a multiple of 256 the
  * two forwards run as ONE pass over two copies of the batch (rows of the second copy take
  * -eps z); every kernel works row by row or sequence by sequence, so the losses are the ones two
- * separate passes give, bit for bit, when both use the same token tile (B*S >= 256).
+ * separate passes give, bit for bit.
+ * From the second call with the same (B, S) on, the step's launch sequence is replayed from a CUDA graph
+ * recorded once (its kernels read seed, eps, lr and clip from device memory and the tokens from the model's
+ * own buffers); results are bit-identical to the direct launches.  See qzo_use_recorded_steps.
  * h_out (may be NULL): {l+, l-, d, d'}; when
  * non-NULL the call synchronises the stream.  The scales are left untouched (the update coefficient is
  * forced to zero on the device) and, when h_out is given, an error is returned if
@@ -224,6 +227,14 @@ int qzo_update_scales(qzo_model* m, uint64_t seed, float lr, float g, float clip
  * The last two are sticky (status word, see qzo_device_status). */
 int qzo_step(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S,
              uint64_t seed, float eps, float lr, float clip, float* h_out);
+
+/* Recorded steps (CUDA graphs) of qzo_step / qzo_step_host: on != 0 (the default) allows them, 0 makes every
+ * step issue its launches directly.  They are bypassed anyway while joint mode, a debug capture or the per-GEMM
+ * timing is on, and switched off for good if recording ever fails. */
+int qzo_use_recorded_steps(qzo_model* m, int on);
+/* *h_count = number of batch shapes whose step is recorded at the moment, or -1 when recorded steps are
+ * switched off (by qzo_use_recorded_steps, or because recording failed). */
+int qzo_recorded_step_count(qzo_model* m, int* h_count);
 
 /* The two halves of qzo_step, for data-parallel replicas (every rank holds the same theta_bar and Delta
  * and its own part of the batch; z depends on (seed, index) only, Sec. 3.1, so ranks exchange losses,
@@ -304,7 +315,8 @@ int qzo_debug_set_status(qzo_model* m, int value);
 int qzo_profile_gemms(qzo_model* m, int max_launches);
 int qzo_profile_read(qzo_model* m, int64_t* launches, double* total_ms, double* total_flops);
 
-/* Number of kernels the library launched since the process started (for benchmark accounting). */
+/* Number of kernels the library launched since the process started, those of replayed recorded steps
+ * included (for benchmark accounting). */
 int64_t qzo_launch_count(void);
 
 #ifdef __cplusplus

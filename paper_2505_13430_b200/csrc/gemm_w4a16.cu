@@ -93,7 +93,8 @@ struct GemmParams {
   int kb_per_split;               // even number of k-blocks per K slice
   int splits, m_tiles, total_units;
   unsigned long long seed;
-  float sign_eps;                 // sign * eps (0 when unperturbed)
+  float sign_eps;                 // sign * eps (0 when unperturbed); with `sp`: the sign alone
+  const StepParams* sp;           // non-null: seed and eps are read from here (a recorded step)
   int pair_rows;                  // > 0: token rows from this one on take -sign_eps (both passes of a step in one launch)
   int* status;
   long long wait_limit;           // cycles after which a device-side wait gives up
@@ -666,6 +667,9 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     // ------------------------------------------------------------------ scale warps
     if (DEQUANT) {
       const int sw = warp - kFirstScaleWarp;
+      // seed and eps of the launch: its own, or those of the recorded step it belongs to
+      const uint64_t seed = p.sp ? (uint64_t)p.sp->seed : p.seed;
+      const float sign_eps = p.sp ? p.sign_eps * p.sp->eps : p.sign_eps;
       int gig = 0;                        // quantisation groups visited by this CTA so far (all units)
       for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x) {
         const Unit w = decode_unit(p, u, TOK);
@@ -681,7 +685,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
           const int row0 = LUT ? w.kb_begin + 2 * gi : (w.kb_begin >> 1) + gi;
           const int rows = LUT ? min(2, w.nkb - 2 * gi) : 1;
           // token tiles never straddle pair_rows (checked on the host)
-          const float se = (p.pair_rows > 0 && w.tok0 >= p.pair_rows) ? -p.sign_eps : p.sign_eps;
+          const float se = (p.pair_rows > 0 && w.tok0 >= p.pair_rows) ? -sign_eps : sign_eps;
           // z does not depend on the stored scales: it is ready before they land
           float z[kScaleRows][4];
           uint2 raw[kScaleRows];
@@ -690,9 +694,9 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             z[j][0] = z[j][1] = z[j][2] = z[j][3] = 0.0f;
             raw[j] = make_uint2(0u, 0u);
             if (live && j < rows) {
-              if (p.sign_eps != 0.0f) {
+              if (sign_eps != 0.0f) {
                 const uint64_t i0 = L.idx_base + (uint64_t)(row0 + j) * (uint64_t)L.N + (uint64_t)(w.n0 + r0);
-                normals_of_block(p.seed, i0 >> 2, z[j]);
+                normals_of_block(seed, i0 >> 2, z[j]);
               }
               if (!Plan::kRawViaCopy) raw[j] = *reinterpret_cast<const uint2*>(L.scales + (size_t)(row0 + j) * L.N + w.n0 + r0);
             }
@@ -1145,9 +1149,10 @@ size_t gemm_workspace_bytes(int M, int K, int N, int pair_rows) {
 // see paired_rows_ok for the row counts that allow it.
 // lut16 (host, 16 floats) non-null: table mode: the nibbles index that table and the scales are [ceil(K/64)][N], one
 // row per block of 64 k; null: int4 with one row of scales per group of 128 k.
+// d_sp (device) non-null: seed and eps are read from it when the kernel runs, the arguments of those names are ignored.
 int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const GemmLinear* lins, int n_lin,
                                 uint64_t seed, int sign, float eps, int pair_rows, void* d_ws, size_t ws_bytes,
-                                int* d_status, cudaStream_t st, const float* lut16) {
+                                int* d_status, cudaStream_t st, const float* lut16, const StepParams* d_sp) {
   if (M <= 0 || K <= 0 || (K % 8) != 0 || n_lin < 1 || n_lin > kMaxGroupedLinears) return QZO_ERR_BAD_ARG;
   if (pair_rows != 0 && !paired_rows_ok(M, pair_rows)) return QZO_ERR_BAD_ARG;
   for (int j = 0; j < n_lin; ++j)
@@ -1164,7 +1169,7 @@ int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const Ge
     if (any_split) {
       for (int j = 0; j < n_lin; ++j)
         QZO_TRY(launch_perturbed_gemm_group(d_x, M, K, lins + j, 1, seed, sign, eps, pair_rows, d_ws, ws_bytes, d_status,
-                                            st, lut16));
+                                            st, lut16, d_sp));
       return QZO_OK;
     }
   }
@@ -1176,7 +1181,8 @@ int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const Ge
   p.num_kb = ceil_div(K, kBlockK);
   p.m_tiles = ceil_div(M, tok);
   p.seed = seed;
-  p.sign_eps = (float)sign * eps;
+  p.sign_eps = d_sp ? (float)sign : (float)sign * eps;
+  p.sp = d_sp;
   p.pair_rows = pair_rows;
   p.status = d_status;
   p.wait_limit = g_debug_wait_limit > 0 ? g_debug_wait_limit : kWaitLimitCycles;

@@ -24,8 +24,10 @@ int launch_relu(__nv_bfloat16* x, int64_t n, cudaStream_t st);
 int launch_cross_entropy(const float* logits, const int32_t* labels, int T, int V, float* row_loss, float* loss,
                          float* sum_out, float* count_out, cudaStream_t st);
 // sums4 = {sum l+, sum l-, kept tokens (+), kept tokens (-)}; out7 = {l+, l-, d, d', lr d' or 0, status, lr_dense d' or 0}
+// sp (device, or null): eps, lr, lr_dense and clip are read from it by the kernel instead of the arguments
 int launch_ddc(const float* sums4, float eps, float lr, float lr_dense, float clip, const int* status, float* out7,
-               cudaStream_t st);
+               cudaStream_t st, const StepParams* sp = nullptr);
+int launch_set_step_params(StepParams* d_sp, uint64_t seed, float eps, float lr, float lr_dense, float clip, cudaStream_t st);
 
 // gemm_w4a16.cu
 constexpr int kMaxSplitTokens = 128;   // token tiles above this never split along K
@@ -45,10 +47,12 @@ struct GemmLinear {
 // pair_rows > 0: rows [0, pair_rows) take sign * eps, rows [pair_rows, M) take -sign * eps, so that one
 // launch serves both passes of a step; allowed when paired_rows_ok(M, pair_rows): pair_rows in {16, 32, 64, 128} or a multiple of 256.
 bool paired_rows_ok(int M, int pair_rows);
-// lut16 (host pointer to 16 floats, or null): table mode, see gemm_w4a16.cu
+// lut16 (host pointer to 16 floats, or null): table mode, see gemm_w4a16.cu; d_sp (device, or null): seed and eps
+// are read from it by the kernel instead of the arguments
 int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const GemmLinear* lins, int n_lin,
                                 uint64_t seed, int sign, float eps, int pair_rows, void* d_ws, size_t ws_bytes,
-                                int* d_status, cudaStream_t st, const float* lut16 = nullptr);
+                                int* d_status, cudaStream_t st, const float* lut16 = nullptr,
+                                const StepParams* d_sp = nullptr);
 // Test hook: later perturbed-GEMM launches of the calling thread use this wait limit (cycles; 0 = the normal
 // one) and withhold the copies of quantisation group `skip_group` of every CTA (-1 = none).
 void set_gemm_wait_debug(long long limit_cycles, int skip_group);

@@ -20,6 +20,7 @@ static std::atomic<long long> g_launches{0};
 void set_last_cuda_error(cudaError_t e) { g_last_cuda_error.store((int)e); }
 int last_cuda_error() { return g_last_cuda_error.load(); }
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+void add_launches(long long n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 long long launch_count() { return g_launches.load(); }
 
 int check_device() {
@@ -126,6 +127,17 @@ struct qzo_model {
   const unsigned long long* vec_base = nullptr;   // device: their logical index bases
   float *vec_plus = nullptr, *vec_minus = nullptr;   // perturbed copies [n_vec][d]
   __nv_bfloat16 *lm_plus = nullptr, *lm_minus = nullptr;   // perturbed copies of the lm_head [V][d]
+  // recorded steps: one CUDA graph per (B, S) of qzo_step; its kernels read seed, eps, lr and clip from sp_dev
+  struct RecordedStep {
+    cudaGraphExec_t exec = nullptr;
+    long long launches = 0;                   // kernels of one replay
+    bool seen = false;                        // the shape ran once the direct way (per-device set-up done)
+  };
+  bool use_graphs = true;
+  std::map<long long, RecordedStep> recorded;
+  cudaStream_t rec_stream = nullptr;          // recording only; nothing ever runs on it
+  qzo::StepParams* sp_dev = nullptr;
+  const qzo::StepParams* cur_sp = nullptr;    // non-null while a step is being recorded
   // optional per-GEMM timing (CUDA events around every perturbed GEMM launch)
   bool profiling = false;
   std::vector<cudaEvent_t> events;
@@ -222,7 +234,7 @@ static int linears(qzo_model* m, const Linear* const* Ls, __nv_bfloat16* const* 
   const bool timed = m->profiling && m->events_used + 2 <= m->events.size();
   if (timed) QZO_CUDA_TRY(cudaEventRecord(m->events[m->events_used], m->stream));
   QZO_TRY(launch_perturbed_gemm_group(in, T, Ls[0]->K, g, n, seed, sign, eps, pair_rows, m->gemm_ws, m->gemm_ws_bytes,
-                                      m->status, m->stream));
+                                      m->status, m->stream, nullptr, m->cur_sp));
   if (timed) {
     QZO_CUDA_TRY(cudaEventRecord(m->events[m->events_used + 1], m->stream));
     m->events_used += 2;
@@ -328,7 +340,7 @@ int check_batch(const qzo_model* m, const void* tok, const void* lab, int B, int
 }
 
 int update_all_scales(qzo_model* m, uint64_t seed, float coef_host, const float* coef_dev) {
-  return launch_update_scales(m->scales, m->flat_entries, seed, 0, coef_host, coef_dev, m->stream);
+  return launch_update_scales(m->scales, m->flat_entries, seed, 0, coef_host, coef_dev, m->stream, m->cur_sp);
 }
 
 // First half of a step: both perturbed forwards (Algorithm 1, the two forward passes on the same batch and
@@ -355,8 +367,8 @@ int step_begin(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, i
 
 // Second half: d, d' (Eq. 6) and the seeded update from the loss sums, all on the device.  With h_out the
 // stream is synchronised and what the device found is reported; the scales are untouched in every error case.
-int step_finish(qzo_model* m, const float* d_sums, uint64_t seed, float eps, float lr, float clip, float* h_out) {
-  QZO_TRY(launch_ddc(d_sums, eps, lr, m->joint ? m->lr_dense : 0.0f, clip, m->status, m->out7, m->stream));
+static int step_finish_launches(qzo_model* m, const float* d_sums, uint64_t seed, float eps, float lr, float clip) {
+  QZO_TRY(launch_ddc(d_sums, eps, lr, m->joint ? m->lr_dense : 0.0f, clip, m->status, m->out7, m->stream, m->cur_sp));
   QZO_TRY(update_all_scales(m, seed, 0.0f, m->out7 + 4));
   if (m->joint) {
     // ZO-SGD on the un-quantised tensors with the same clipped d' and the same z stream (Def. 3.2)
@@ -367,7 +379,12 @@ int step_finish(qzo_model* m, const float* d_sums, uint64_t seed, float eps, flo
     QZO_TRY(launch_update_vectors(const_cast<float* const*>(reinterpret_cast<const float* const*>(m->vec_table)), m->vec_base,
                                   m->n_vec, m->desc.d_model, seed, coef, m->stream));
   }
-  if (h_out) {
+  return QZO_OK;
+}
+
+// What the device found in the step just launched (synchronises the stream): l+, l-, d, d' and the error, if any.
+static int read_step_result(qzo_model* m, float* h_out) {
+  {
     float host[6];
     QZO_CUDA_TRY(cudaMemcpyAsync(host, m->out7, sizeof(host), cudaMemcpyDeviceToHost, m->stream));
     QZO_CUDA_TRY(cudaStreamSynchronize(m->stream));
@@ -380,8 +397,74 @@ int step_finish(qzo_model* m, const float* d_sums, uint64_t seed, float eps, flo
   return QZO_OK;
 }
 
+int step_finish(qzo_model* m, const float* d_sums, uint64_t seed, float eps, float lr, float clip, float* h_out) {
+  QZO_TRY(step_finish_launches(m, d_sums, seed, eps, lr, clip));
+  return h_out ? read_step_result(m, h_out) : QZO_OK;
+}
+
+// Records the launch sequence of a whole step on (B, S) into a CUDA graph.  The step's kernels take seed, eps,
+// lr and clip from m->sp_dev and its tokens from the model's own buffers, so the graph serves every later step
+// of that shape.  Nothing runs while recording.  A failure ends the recording and switches recorded steps off.
+static int record_step(qzo_model* m, int B, int S, qzo_model::RecordedStep* rec) {
+  const long long before = launch_count();
+  // recorded on a stream of the model's own (the caller's may be the legacy default stream, which cannot
+  // record); the graph is then launched on the caller's stream
+  if (m->rec_stream == nullptr && cudaStreamCreateWithFlags(&m->rec_stream, cudaStreamNonBlocking) != cudaSuccess) {
+    (void)cudaGetLastError();
+    m->rec_stream = nullptr;
+    return QZO_ERR_CUDA;
+  }
+  if (cudaStreamBeginCapture(m->rec_stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return QZO_ERR_CUDA;
+  }
+  cudaStream_t const callers = m->stream;
+  m->stream = m->rec_stream;
+  m->cur_sp = m->sp_dev;
+  int rc = step_begin(m, m->tok_dev, m->lab_dev, B, S, 0, 1.0f, m->sums);
+  if (rc == QZO_OK) rc = step_finish_launches(m, m->sums, 0, 1.0f, 0.0f, 0.0f);
+  m->cur_sp = nullptr;
+  m->stream = callers;
+  cudaGraph_t graph = nullptr;
+  const cudaError_t e = cudaStreamEndCapture(m->rec_stream, &graph);
+  if (rc == QZO_OK && (e != cudaSuccess || graph == nullptr)) rc = QZO_ERR_CUDA;
+  if (rc == QZO_OK && cudaGraphInstantiate(&rec->exec, graph, 0) != cudaSuccess) rc = QZO_ERR_CUDA;
+  if (graph) cudaGraphDestroy(graph);
+  rec->launches = launch_count() - before;
+  add_launches(-rec->launches);             // recorded, not run: a replay counts them
+  if (rc != QZO_OK) {
+    (void)cudaGetLastError();
+    rec->exec = nullptr;
+    return rc;
+  }
+  return QZO_OK;
+}
+
 int step_device(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S, uint64_t seed, float eps,
                 float lr, float clip, float* h_out) {
+  // A step whose launch sequence depends on nothing but (B, S) is recorded once and replayed: with few tokens
+  // the host would otherwise need longer to issue the step's launches than the device needs to run them.
+  const bool replay = m->use_graphs && !m->joint && m->capture_layer < 0 && !m->profiling;
+  if (replay) {
+    qzo_model::RecordedStep& rec = m->recorded[((long long)B << 32) | (long long)S];
+    if (rec.seen) {
+      const size_t bytes = (size_t)B * S * sizeof(int32_t);
+      if (d_tokens != m->tok_dev)
+        QZO_CUDA_TRY(cudaMemcpyAsync(m->tok_dev, d_tokens, bytes, cudaMemcpyDeviceToDevice, m->stream));
+      if (d_labels != m->lab_dev)
+        QZO_CUDA_TRY(cudaMemcpyAsync(m->lab_dev, d_labels, bytes, cudaMemcpyDeviceToDevice, m->stream));
+      if (rec.exec == nullptr && record_step(m, B, S, &rec) != QZO_OK) m->use_graphs = false;
+      if (rec.exec != nullptr) {
+        QZO_TRY(launch_set_step_params(m->sp_dev, seed, eps, lr, 0.0f, clip, m->stream));
+        QZO_CUDA_TRY(cudaGraphLaunch(rec.exec, m->stream));
+        add_launches(rec.launches);
+        return h_out ? read_step_result(m, h_out) : QZO_OK;
+      }
+      d_tokens = m->tok_dev;
+      d_labels = m->lab_dev;
+    }
+    rec.seen = true;                          // the first step of a shape runs the direct way
+  }
   QZO_TRY(step_begin(m, d_tokens, d_labels, B, S, seed, eps, m->sums));
   return step_finish(m, m->sums, seed, eps, lr, clip, h_out);
 }
@@ -639,6 +722,7 @@ int qzo_init_model(const qzo_model_desc* desc, const qzo_tensor* tensors, int n_
   m->sums = scal + 4;         // [4..7]
   m->out7 = scal + 8;         // [8..14]
   m->status = (int*)(scal + 32);
+  m->sp_dev = reinterpret_cast<StepParams*>(scal + 40);
   m->rope_cs = (float*)(ws + p.off_rope);
   m->tok_dev = (int32_t*)(ws + p.off_tok);
   m->lab_dev = (int32_t*)(ws + p.off_lab);
@@ -689,6 +773,9 @@ int qzo_profile_read(qzo_model* m, int64_t* launches, double* total_ms, double* 
 int qzo_free_model(qzo_model* m) {
   if (!m) return QZO_ERR_BAD_ARG;
   for (cudaEvent_t e : m->events) cudaEventDestroy(e);
+  for (auto& kv : m->recorded)
+    if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);
+  if (m->rec_stream) cudaStreamDestroy(m->rec_stream);
   delete m;
   return QZO_OK;
 }
@@ -712,6 +799,20 @@ int qzo_step(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int
   QZO_TRY(check_batch(m, d_tokens, d_labels, B, S));
   if (!(eps > 0.0f) || !(clip >= 0.0f) || !std::isfinite(lr)) return QZO_ERR_BAD_ARG;
   return step_device(m, d_tokens, d_labels, B, S, seed, eps, lr, clip, h_out);
+}
+
+int qzo_use_recorded_steps(qzo_model* m, int on) {
+  if (!m) return QZO_ERR_BAD_ARG;
+  m->use_graphs = on != 0;
+  return QZO_OK;
+}
+
+int qzo_recorded_step_count(qzo_model* m, int* h_count) {
+  if (!m || !h_count) return QZO_ERR_BAD_ARG;
+  int n = 0;
+  for (const auto& kv : m->recorded) n += kv.second.exec != nullptr;
+  *h_count = m->use_graphs ? n : -1;
+  return QZO_OK;
 }
 
 int qzo_step_host(qzo_model* m, const int32_t* h_tokens, const int32_t* h_labels, int B, int S, uint64_t seed,

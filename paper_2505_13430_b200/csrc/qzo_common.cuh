@@ -33,6 +33,13 @@ void set_last_cuda_error(cudaError_t e);
 constexpr int kStatusTimeout = 1;    // a bounded device-side wait expired in some launch
 constexpr int kStatusBadToken = 2;   // a token id outside [0, vocab) reached the embedding
 
+// Per-step quantities of a recorded step (a CUDA graph that is replayed): its kernels read them from
+// device memory, so that one recorded launch sequence serves every seed and every step size.
+struct StepParams {
+  unsigned long long seed;
+  float eps, lr, lr_dense, clip;
+};
+
 constexpr int kGroup = 128;          // rows of one quantisation group (paper: group 128)
 constexpr int kTileN = 128;          // output features per GEMM tile (UMMA M)
 constexpr int kBlockK = 64;          // K elements per pipeline stage (one 128-byte swizzle atom of bf16)

@@ -27,7 +27,7 @@ EXPORTS = (
     "qzo_scale_layout", "qzo_workspace_bytes", "qzo_init_model", "qzo_free_model", "qzo_forward_loss",
     "qzo_update_scales", "qzo_step", "qzo_step_host", "qzo_debug_set_capture", "qzo_debug_layer_output",
     "qzo_device_status", "qzo_launch_count", "qzo_profile_gemms", "qzo_profile_read",
-    "qzo_step_begin", "qzo_step_finish", "qzo_get_scales", "qzo_set_scales", "qzo_debug_set_status",
+    "qzo_step_begin", "qzo_step_finish", "qzo_get_scales", "qzo_set_scales", "qzo_debug_set_status", "qzo_use_recorded_steps", "qzo_recorded_step_count",
     "qzo_joint_workspace_bytes", "qzo_enable_joint_spsa", "qzo_perturbed_gemm_table16", "qzo_debug_gemm_wait_expiry",
 )
 
@@ -92,6 +92,8 @@ def _load():
         "qzo_get_scales": (ci, [vp, ci, vp, sz]),
         "qzo_set_scales": (ci, [vp, ci, vp, sz]),
         "qzo_debug_set_status": (ci, [vp, ci]),
+        "qzo_use_recorded_steps": (ci, [vp, ci]),
+        "qzo_recorded_step_count": (ci, [vp, vp]),
         "qzo_joint_workspace_bytes": (ci, [P(ModelDesc), P(sz)]),
         "qzo_enable_joint_spsa": (ci, [vp, vp, sz, cf]),
         "qzo_debug_set_capture": (ci, [vp, ci]),
@@ -390,6 +392,14 @@ class Model:
 
     def qzo_debug_set_status(self, value):
         _check(_lib.qzo_debug_set_status(self.handle, value), "qzo_debug_set_status")
+
+    def qzo_use_recorded_steps(self, on):
+        _check(_lib.qzo_use_recorded_steps(self.handle, 1 if on else 0), "qzo_use_recorded_steps")
+
+    def qzo_recorded_step_count(self):
+        n = ctypes.c_int(0)
+        _check(_lib.qzo_recorded_step_count(self.handle, ctypes.byref(n)), "qzo_recorded_step_count")
+        return n.value
 
     def qzo_step_host(self, tokens_host, labels_host, seed, eps, lr, clip):
         assert not tokens_host.is_cuda and tokens_host.dtype == torch.int32 and tokens_host.is_contiguous()
