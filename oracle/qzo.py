@@ -1,12 +1,13 @@
 """One QZO step (oracle): Algorithm 1, Eq. 5 (Q-SPSA) and Eq. 6 (DDC).
 
-Two forms are given.  `step_literal` is the in-place form of Algorithm 1: the
-scales themselves are moved by +eps z before the first forward, by -2 eps z
-before the second and by +eps z afterwards (which restores them), then d, d'
-and the seeded update with max(., 0) follow.  `step_functional` evaluates the
-same quantities from the untouched scales, Delta' = Delta + sign*eps*z, which
-is what the library does.  In exact arithmetic they agree; the tests require
-agreement to fp64 rounding (the equivalence is the property being pinned).
+`step_functional` evaluates both losses from the untouched scales,
+Delta' = Delta + sign*eps*z (Eq. 5), then d, d' (Eq. 6) and the seeded update
+with max(., 0) (Algorithm 1's last loop); this is also what the library does.
+Algorithm 1 itself moves the scales in place (by +eps z, then -2 eps z, then
++eps z to restore them); `perturb_scales_in_place` is that single operation,
+kept so that the tests can pin the equivalence of the two readings: a forward
+on scales moved in place equals the forward with the matching sign, and the
+three moves return the scales to where they started.
 
 Storage rounding of the updated scale (bf16, ties to even) is a reading: the
 paper does not fix the dtype of Delta.  `lr * d'` is formed once in fp32 and
@@ -104,8 +105,9 @@ def step_functional(model, tokens, labels, seed, eps, lr, C, update=True, joint=
     return lp, lm, d, dc
 
 
-def _perturb_in_place(model, scale, seed):
-    """PERTURB_SCALES(Delta, scale, s): Delta_i += scale * z_i, fp64, no clamp."""
+def perturb_scales_in_place(model, scale, seed):
+    """Delta_i += scale * z_i(seed) for every scale of the model, in fp64, without clamping
+    (the in-place perturbation of Algorithm 1; the scales become fp64 arrays)."""
     cfg = model["cfg"]
     bases, _ = scale_index_bases(cfg)
     for li, layer in enumerate(model["layers"]):
@@ -114,26 +116,3 @@ def _perturb_in_place(model, scale, seed):
             s = np.asarray(p["s"], dtype=np.float64)
             z = philox.normal_range(seed, bases[li][name], s.size).astype(np.float64)
             p["s"] = s + scale * z.reshape(s.shape)
-
-
-def step_literal(model, tokens, labels, seed, eps, lr, C):
-    """Algorithm 1 in its in-place form, scales held in fp64 and mutated.
-
-    Returns (l+, l-, d, d'); the model's scales end as fp64
-    max(Delta_i - lr d' z_i, 0) without storage rounding.
-    """
-    _perturb_in_place(model, +eps, seed)
-    lp = forward_loss(model, tokens, labels, seed, 0, eps)
-    _perturb_in_place(model, -2.0 * eps, seed)
-    lm = forward_loss(model, tokens, labels, seed, 0, eps)
-    _perturb_in_place(model, +eps, seed)
-    d = directional_derivative(lp, lm, eps)
-    dc = ddc_clip(d, C)
-    cfg = model["cfg"]
-    bases, _ = scale_index_bases(cfg)
-    for li, layer in enumerate(model["layers"]):
-        for name in LINEAR_ORDER[cfg["arch"]]:
-            p = layer["lin"][name]
-            z = philox.normal_range(seed, bases[li][name], p["s"].size).astype(np.float64)
-            p["s"] = np.maximum(p["s"] - lr * dc * z.reshape(p["s"].shape), 0.0)
-    return lp, lm, d, dc

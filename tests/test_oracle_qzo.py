@@ -1,5 +1,5 @@
 """Pins for oracle/qzo.py: Eq. 6 cases, the exact finite difference on a quadratic loss,
-Algorithm 1 literal vs functional, and the update's invariants."""
+Algorithm 1's in-place perturbations against the functional form, and the update's invariants."""
 import numpy as np
 
 from oracle import int4, linear, philox, qzo, model as omodel
@@ -70,20 +70,33 @@ def test_cross_entropy_difference_converges_quadratically():
     assert e1 > 0 and 2.5 < e1 / e2 < 6.5 and e3 < e2
 
 
-def test_literal_algorithm1_equals_functional_form():
+def test_in_place_perturbation_equals_functional_form():
+    # Algorithm 1 moves the scales in place; the oracle (and the library) evaluate Delta + sign*eps*z from the
+    # untouched scales.  The two readings agree: a forward on scales moved by +eps z (then by -2 eps z) is the
+    # forward with sign +1 (-1), and the third move restores the scales to fp64 rounding.
     cfg, m, tok, lab = _setup()
-    seed, eps, lr, C = 42, 1e-3, 1e-3, 100.0
+    seed, eps = 42, 1e-3
     a, b = clone_model(m), clone_model(m)
-    lp, lm, d, dc = qzo.step_functional(a, tok, lab, seed, eps, lr, C, update=False)
-    lp2, lm2, d2, dc2 = qzo.step_literal(b, tok, lab, seed, eps, lr, C)
-    assert abs(lp - lp2) < 1e-12 and abs(lm - lm2) < 1e-12 and abs(d - d2) < 1e-8
-    # updated scales: literal fp64 result vs functional fp32+bf16 result
-    qzo.update_model_scales(a, seed, lr, dc)
+    lp = omodel.forward_loss(a, tok, lab, seed, +1, eps)
+    lm = omodel.forward_loss(a, tok, lab, seed, -1, eps)
+    qzo.perturb_scales_in_place(b, +eps, seed)
+    assert abs(omodel.forward_loss(b, tok, lab, seed, 0, eps) - lp) < 1e-12
+    qzo.perturb_scales_in_place(b, -2.0 * eps, seed)
+    assert abs(omodel.forward_loss(b, tok, lab, seed, 0, eps) - lm) < 1e-12
+    qzo.perturb_scales_in_place(b, +eps, seed)
+    moved = False
     for la, lb in zip(a["layers"], b["layers"]):
         for name in la["lin"]:
-            sa, sb = la["lin"][name]["s"].astype(np.float64), lb["lin"][name]["s"]
-            assert np.all(sb >= 0) and np.all(sa >= 0)
-            assert np.all(np.abs(sa - sb) <= 2.0 ** -8 * np.abs(sb) + 1e-12)     # bf16 storage rounding only
+            sa, sb = np.asarray(la["lin"][name]["s"], dtype=np.float64), lb["lin"][name]["s"]
+            assert np.all(np.abs(sa - sb) <= 1e-15)
+            moved = moved or sb.dtype == np.float64
+    assert moved and lp != lm
+    # the step built on the functional form: d from those two losses, d' clipped, scales updated and non-negative
+    out = qzo.step_functional(a, tok, lab, seed, eps, 1e-3, 100.0)
+    assert out[0] == lp and out[1] == lm and out[2] == qzo.directional_derivative(lp, lm, eps)
+    for la in a["layers"]:
+        for name in la["lin"]:
+            assert np.all(la["lin"][name]["s"] >= 0)
 
 
 def test_update_invariants():
