@@ -124,8 +124,16 @@ def test_truncated_full_width_step_losses_match_oracle(lib, workload, n_layers):
     cfg, om, gm = _oracle_and_gpu_model(lib, workload, n_layers, B * S)
     tok, lab = inputs.tokens_and_labels(cfg, B, S, seed=7)
     seed, eps = 42, c["eps"]
+    before = gm.scales.clone()
     lp, lm, d, dc = gm.qzo_step(tok.cuda(), lab.cuda(), seed, eps, c["lr"], c["clip"])
     assert gm.qzo_device_status() == 0
+    # the same step again, recorded into a CUDA graph and then replayed: bit-identical at the full width too
+    after = gm.scales.clone()
+    for _ in range(2):
+        gm.scales.copy_(before)
+        assert gm.qzo_step(tok.cuda(), lab.cuda(), seed, eps, c["lr"], c["clip"]) == (lp, lm, d, dc)
+        assert torch.equal(gm.scales.view(torch.int16), after.view(torch.int16))
+    assert gm.qzo_recorded_step_count() == 1
     rp = omodel.forward_loss(om, tok.numpy(), lab.numpy(), seed, +1, eps)
     rm = omodel.forward_loss(om, tok.numpy(), lab.numpy(), seed, -1, eps)
     d_ref = (rp - rm) / (2 * eps)
