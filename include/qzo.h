@@ -230,7 +230,8 @@ int qzo_step(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int
 
 /* Recorded steps (CUDA graphs) of qzo_step / qzo_step_host: on != 0 (the default) allows them, 0 makes every
  * step issue its launches directly.  They are bypassed anyway while joint mode, a debug capture or the per-GEMM
- * timing is on, and switched off for good if recording ever fails. */
+ * timing is on, for batch shapes beyond the first 16 a model has seen, and switched off for good if recording
+ * ever fails. */
 int qzo_use_recorded_steps(qzo_model* m, int on);
 /* *h_count = number of batch shapes whose step is recorded at the moment, or -1 when recorded steps are
  * switched off (by qzo_use_recorded_steps, or because recording failed). */

@@ -131,6 +131,7 @@ struct qzo_model {
   struct RecordedStep {
     cudaGraphExec_t exec = nullptr;
     long long launches = 0;                   // kernels of one replay
+    int rows = 0;                             // token rows of the step's forward (what last_T is after it)
     bool seen = false;                        // the shape ran once the direct way (per-device set-up done)
   };
   bool use_graphs = true;
@@ -402,6 +403,8 @@ int step_finish(qzo_model* m, const float* d_sums, uint64_t seed, float eps, flo
   return h_out ? read_step_result(m, h_out) : QZO_OK;
 }
 
+constexpr size_t kMaxRecordedShapes = 16;
+
 // Records the launch sequence of a whole step on (B, S) into a CUDA graph.  The step's kernels take seed, eps,
 // lr and clip from m->sp_dev and its tokens from the model's own buffers, so the graph serves every later step
 // of that shape.  Nothing runs while recording.  A failure ends the recording and switches recorded steps off.
@@ -431,6 +434,7 @@ static int record_step(qzo_model* m, int B, int S, qzo_model::RecordedStep* rec)
   if (rc == QZO_OK && cudaGraphInstantiate(&rec->exec, graph, 0) != cudaSuccess) rc = QZO_ERR_CUDA;
   if (graph) cudaGraphDestroy(graph);
   rec->launches = launch_count() - before;
+  rec->rows = m->last_T;
   add_launches(-rec->launches);             // recorded, not run: a replay counts them
   if (rc != QZO_OK) {
     (void)cudaGetLastError();
@@ -444,9 +448,12 @@ int step_device(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, 
                 float lr, float clip, float* h_out) {
   // A step whose launch sequence depends on nothing but (B, S) is recorded once and replayed: with few tokens
   // the host would otherwise need longer to issue the step's launches than the device needs to run them.
-  const bool replay = m->use_graphs && !m->joint && m->capture_layer < 0 && !m->profiling;
+  const long long shape = ((long long)B << 32) | (long long)S;
+  // at most kMaxRecordedShapes batch shapes are recorded per model; further shapes run the direct way
+  const bool replay = m->use_graphs && !m->joint && m->capture_layer < 0 && !m->profiling &&
+                      (m->recorded.size() < kMaxRecordedShapes || m->recorded.count(shape) > 0);
   if (replay) {
-    qzo_model::RecordedStep& rec = m->recorded[((long long)B << 32) | (long long)S];
+    qzo_model::RecordedStep& rec = m->recorded[shape];
     if (rec.seen) {
       const size_t bytes = (size_t)B * S * sizeof(int32_t);
       if (d_tokens != m->tok_dev)
@@ -458,6 +465,7 @@ int step_device(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, 
         QZO_TRY(launch_set_step_params(m->sp_dev, seed, eps, lr, 0.0f, clip, m->stream));
         QZO_CUDA_TRY(cudaGraphLaunch(rec.exec, m->stream));
         add_launches(rec.launches);
+        m->last_T = rec.rows;
         return h_out ? read_step_result(m, h_out) : QZO_OK;
       }
       d_tokens = m->tok_dev;

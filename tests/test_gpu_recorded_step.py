@@ -41,6 +41,13 @@ def test_replayed_steps_equal_direct_steps(name):
         assert torch.equal(recorded.scales.view(torch.int16), direct.scales.view(torch.int16)), (nb, ns, seed)
         # a replay accounts for the kernels it runs (plus the one that writes the step's parameters)
         assert n1 - n0 in (n2 - n1, n2 - n1 + 1), (n1 - n0, n2 - n1)
+        # the logits both models keep from the step's forward (both signs' rows when they ran as one pass)
+        rows = nb * ns * (2 if nb * ns in (16, 32, 64, 128) or (nb * ns) % 256 == 0 else 1)
+        la = recorded.qzo_debug_layer_output(0, 1, rows)
+        lb = direct.qzo_debug_layer_output(0, 1, rows)
+        assert torch.equal(la.view(torch.int32), lb.view(torch.int32)), (nb, ns, seed)
+        with pytest.raises(qzo.QzoError):
+            recorded.qzo_debug_layer_output(0, 1, rows - 1)           # the buffer must hold every row of the last forward
     # every shape was recorded on one model and none on the other; the host-token entry point takes the same route
     assert recorded.qzo_recorded_step_count() == len(shapes) and direct.qzo_recorded_step_count() == -1
     assert recorded.qzo_device_status() == 0 and direct.qzo_device_status() == 0
@@ -74,5 +81,22 @@ def test_replayed_step_reports_failures_and_leaves_the_scales_untouched():
     assert e.value.status == qzo.ERR_NONFINITE
     torch.cuda.synchronize()
     assert bool((recorded.scales.view(torch.int16) == before.view(torch.int16)).all())
+    recorded.close()
+    direct.close()
+
+
+def test_shapes_beyond_the_recording_limit_run_directly():
+    # A model records at most 16 batch shapes; the shapes it meets after that keep running launch by launch,
+    # with the same results.
+    qzo, c, recorded, direct, tok, lab = _models("tiny")
+    shapes = [(nb, ns) for nb in (1, 2, 3) for ns in (8, 16, 24, 32, 40, 48)]           # 18 shapes
+    for rep in range(2):
+        for i, (nb, ns) in enumerate(shapes):
+            t, l = tok[:nb, :ns].contiguous().cuda(), lab[:nb, :ns].contiguous().cuda()
+            a = recorded.qzo_step(t, l, 50 + i, c["eps"], c["lr"] * 50, c["clip"])
+            b = direct.qzo_step(t, l, 50 + i, c["eps"], c["lr"] * 50, c["clip"])
+            assert a == b, (nb, ns)
+    assert recorded.qzo_recorded_step_count() == 16
+    assert torch.equal(recorded.scales.view(torch.int16), direct.scales.view(torch.int16))
     recorded.close()
     direct.close()
