@@ -215,9 +215,9 @@ int qzo_update_scales(qzo_model* m, uint64_t seed, float lr, float g, float clip
  * two forwards run as ONE pass over two copies of the batch (rows of the second copy take
  * -eps z); every kernel works row by row or sequence by sequence, so the losses are the ones two
  * separate passes give, bit for bit.
- * From the second call with the same (B, S) on, the step's launch sequence is replayed from a CUDA graph
- * recorded once (its kernels read seed, eps, lr and clip from device memory and the tokens from the model's
- * own buffers); results are bit-identical to the direct launches.  See qzo_use_recorded_steps.
+ * From the second call with the same (B, S) on, the launch sequence of the two forwards is replayed from a CUDA
+ * graph recorded once (its GEMMs read seed and eps from device memory, the tokens come from the model's own
+ * buffers); results are bit-identical to the direct launches.  See qzo_use_recorded_steps.
  * h_out (may be NULL): {l+, l-, d, d'}; when
  * non-NULL the call synchronises the stream.  The scales are left untouched (the update coefficient is
  * forced to zero on the device) and, when h_out is given, an error is returned if
@@ -228,7 +228,7 @@ int qzo_update_scales(qzo_model* m, uint64_t seed, float lr, float g, float clip
 int qzo_step(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S,
              uint64_t seed, float eps, float lr, float clip, float* h_out);
 
-/* Recorded steps (CUDA graphs) of qzo_step / qzo_step_host: on != 0 (the default) allows them, 0 makes every
+/* Recorded steps (CUDA graphs) of qzo_step / qzo_step_host / qzo_step_begin: on != 0 (the default) allows them, 0 makes every
  * step issue its launches directly.  They are bypassed anyway while joint mode, a debug capture or the per-GEMM
  * timing is on, for batch shapes beyond the first 16 a model has seen, and switched off for good if recording
  * ever fails. */

@@ -27,9 +27,8 @@ int launch_unpack(const uint32_t* d_packed, int K, int N, int8_t* d_q, cudaStrea
 size_t repacked_bytes(int K, int N);
 int launch_repack(const uint32_t* d_packed, int K, int N, void* d_out, cudaStream_t st);
 int launch_unpack_kernel_layout(const void* d_wq, int K, int N, int8_t* d_q, cudaStream_t st);
-// sp (device, or null): the seed is read from it by the kernel instead of the argument
 int launch_update_scales(__nv_bfloat16* d_s, int64_t count, uint64_t seed, uint64_t index_base,
-                         float coef_host, const float* coef_dev, cudaStream_t st, const StepParams* sp = nullptr);
+                         float coef_host, const float* coef_dev, cudaStream_t st);
 // joint mode: plain SPSA on the un-quantised tensors
 int launch_perturb_dense_bf16(const __nv_bfloat16* src, __nv_bfloat16* dst, int64_t count, uint64_t seed,
                               uint64_t index_base, float sign_eps, cudaStream_t st);

@@ -476,8 +476,7 @@ __global__ void ce_mean_kernel(const float* __restrict__ row_loss, const int32_t
 // (no update) when a loss is not finite or the status word reports a failed launch or a bad token.
 // out = {l+, l-, d, d', coef, status word as a float, coef of the un-quantised tensors (joint mode)}
 __global__ void ddc_kernel(const float* __restrict__ sums, float eps, float lr, float lr_dense, float clip,
-                           const int* __restrict__ status, float* __restrict__ out, const StepParams* __restrict__ sp) {
-  if (sp) { eps = sp->eps; lr = sp->lr; lr_dense = sp->lr_dense; clip = sp->clip; }
+                           const int* __restrict__ status, float* __restrict__ out) {
   const float a = sums[0] / fmaxf(sums[2], 1.0f), b = sums[1] / fmaxf(sums[3], 1.0f);
   const float d = (a - b) / (2.0f * eps);
   const float dc = fminf(fmaxf(d, -clip), clip);
@@ -489,7 +488,7 @@ __global__ void ddc_kernel(const float* __restrict__ sums, float eps, float lr, 
   out[6] = good ? __fmul_rn(lr_dense, dc) : 0.0f;    // joint mode: step of the un-quantised tensors
 }
 
-// The per-step quantities of a recorded step, written before it is replayed.
+// The per-step quantities of a recorded forward, written before it is replayed.
 __global__ void set_step_params_kernel(StepParams* __restrict__ dst, StepParams v) { *dst = v; }
 
 }  // namespace
@@ -565,12 +564,12 @@ int launch_cross_entropy(const float* logits, const int32_t* labels, int T, int 
   return QZO_OK;
 }
 int launch_ddc(const float* sums4, float eps, float lr, float lr_dense, float clip, const int* status, float* out7,
-               cudaStream_t st, const StepParams* sp) {
-  QZO_LAUNCH(ddc_kernel, dim3(1), dim3(1), 0, st, sums4, eps, lr, lr_dense, clip, status, out7, sp);
+               cudaStream_t st) {
+  QZO_LAUNCH(ddc_kernel, dim3(1), dim3(1), 0, st, sums4, eps, lr, lr_dense, clip, status, out7);
   return QZO_OK;
 }
-int launch_set_step_params(StepParams* d_sp, uint64_t seed, float eps, float lr, float lr_dense, float clip, cudaStream_t st) {
-  QZO_LAUNCH(set_step_params_kernel, dim3(1), dim3(1), 0, st, d_sp, StepParams{seed, eps, lr, lr_dense, clip});
+int launch_set_step_params(StepParams* d_sp, uint64_t seed, float eps, cudaStream_t st) {
+  QZO_LAUNCH(set_step_params_kernel, dim3(1), dim3(1), 0, st, d_sp, StepParams{seed, eps});
   return QZO_OK;
 }
 

@@ -24,10 +24,9 @@ int launch_relu(__nv_bfloat16* x, int64_t n, cudaStream_t st);
 int launch_cross_entropy(const float* logits, const int32_t* labels, int T, int V, float* row_loss, float* loss,
                          float* sum_out, float* count_out, cudaStream_t st);
 // sums4 = {sum l+, sum l-, kept tokens (+), kept tokens (-)}; out7 = {l+, l-, d, d', lr d' or 0, status, lr_dense d' or 0}
-// sp (device, or null): eps, lr, lr_dense and clip are read from it by the kernel instead of the arguments
 int launch_ddc(const float* sums4, float eps, float lr, float lr_dense, float clip, const int* status, float* out7,
-               cudaStream_t st, const StepParams* sp = nullptr);
-int launch_set_step_params(StepParams* d_sp, uint64_t seed, float eps, float lr, float lr_dense, float clip, cudaStream_t st);
+               cudaStream_t st);
+int launch_set_step_params(StepParams* d_sp, uint64_t seed, float eps, cudaStream_t st);
 
 // gemm_w4a16.cu
 constexpr int kMaxSplitTokens = 128;   // token tiles above this never split along K

@@ -127,7 +127,7 @@ struct qzo_model {
   const unsigned long long* vec_base = nullptr;   // device: their logical index bases
   float *vec_plus = nullptr, *vec_minus = nullptr;   // perturbed copies [n_vec][d]
   __nv_bfloat16 *lm_plus = nullptr, *lm_minus = nullptr;   // perturbed copies of the lm_head [V][d]
-  // recorded steps: one CUDA graph per (B, S) of qzo_step; its kernels read seed, eps, lr and clip from sp_dev
+  // recorded steps: one CUDA graph per (B, S) holding a step's two forwards; its GEMMs read seed and eps from sp_dev
   struct RecordedStep {
     cudaGraphExec_t exec = nullptr;
     long long launches = 0;                   // kernels of one replay
@@ -341,7 +341,7 @@ int check_batch(const qzo_model* m, const void* tok, const void* lab, int B, int
 }
 
 int update_all_scales(qzo_model* m, uint64_t seed, float coef_host, const float* coef_dev) {
-  return launch_update_scales(m->scales, m->flat_entries, seed, 0, coef_host, coef_dev, m->stream, m->cur_sp);
+  return launch_update_scales(m->scales, m->flat_entries, seed, 0, coef_host, coef_dev, m->stream);
 }
 
 // First half of a step: both perturbed forwards (Algorithm 1, the two forward passes on the same batch and
@@ -369,7 +369,7 @@ int step_begin(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, i
 // Second half: d, d' (Eq. 6) and the seeded update from the loss sums, all on the device.  With h_out the
 // stream is synchronised and what the device found is reported; the scales are untouched in every error case.
 static int step_finish_launches(qzo_model* m, const float* d_sums, uint64_t seed, float eps, float lr, float clip) {
-  QZO_TRY(launch_ddc(d_sums, eps, lr, m->joint ? m->lr_dense : 0.0f, clip, m->status, m->out7, m->stream, m->cur_sp));
+  QZO_TRY(launch_ddc(d_sums, eps, lr, m->joint ? m->lr_dense : 0.0f, clip, m->status, m->out7, m->stream));
   QZO_TRY(update_all_scales(m, seed, 0.0f, m->out7 + 4));
   if (m->joint) {
     // ZO-SGD on the un-quantised tensors with the same clipped d' and the same z stream (Def. 3.2)
@@ -405,10 +405,11 @@ int step_finish(qzo_model* m, const float* d_sums, uint64_t seed, float eps, flo
 
 constexpr size_t kMaxRecordedShapes = 16;
 
-// Records the launch sequence of a whole step on (B, S) into a CUDA graph.  The step's kernels take seed, eps,
-// lr and clip from m->sp_dev and its tokens from the model's own buffers, so the graph serves every later step
-// of that shape.  Nothing runs while recording.  A failure ends the recording and switches recorded steps off.
-static int record_step(qzo_model* m, int B, int S, qzo_model::RecordedStep* rec) {
+// Records the launch sequence of a step's two forwards on (B, S) into a CUDA graph.  Their GEMMs take seed and eps
+// from m->sp_dev, the tokens come from the model's own buffers and the loss sums go to m->sums, so the graph serves
+// every later step of that shape.  Nothing runs while recording.  A failure ends the recording and switches
+// recorded steps off.
+static int record_forwards(qzo_model* m, int B, int S, qzo_model::RecordedStep* rec) {
   const long long before = launch_count();
   // recorded on a stream of the model's own (the caller's may be the legacy default stream, which cannot
   // record); the graph is then launched on the caller's stream
@@ -425,7 +426,6 @@ static int record_step(qzo_model* m, int B, int S, qzo_model::RecordedStep* rec)
   m->stream = m->rec_stream;
   m->cur_sp = m->sp_dev;
   int rc = step_begin(m, m->tok_dev, m->lab_dev, B, S, 0, 1.0f, m->sums);
-  if (rc == QZO_OK) rc = step_finish_launches(m, m->sums, 0, 1.0f, 0.0f, 0.0f);
   m->cur_sp = nullptr;
   m->stream = callers;
   cudaGraph_t graph = nullptr;
@@ -444,10 +444,11 @@ static int record_step(qzo_model* m, int B, int S, qzo_model::RecordedStep* rec)
   return QZO_OK;
 }
 
-int step_device(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S, uint64_t seed, float eps,
-                float lr, float clip, float* h_out) {
-  // A step whose launch sequence depends on nothing but (B, S) is recorded once and replayed: with few tokens
-  // the host would otherwise need longer to issue the step's launches than the device needs to run them.
+// The two forwards of a step (step_begin), replayed from a recording where there is one.  A launch sequence that
+// depends on nothing but (B, S) is recorded once and replayed: with few tokens the host would otherwise need longer
+// to issue the launches than the device needs to run them.
+int step_begin_replayed(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S, uint64_t seed,
+                        float eps, float* d_sums) {
   const long long shape = ((long long)B << 32) | (long long)S;
   // at most kMaxRecordedShapes batch shapes are recorded per model; further shapes run the direct way
   const bool replay = m->use_graphs && !m->joint && m->capture_layer < 0 && !m->profiling &&
@@ -460,20 +461,27 @@ int step_device(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, 
         QZO_CUDA_TRY(cudaMemcpyAsync(m->tok_dev, d_tokens, bytes, cudaMemcpyDeviceToDevice, m->stream));
       if (d_labels != m->lab_dev)
         QZO_CUDA_TRY(cudaMemcpyAsync(m->lab_dev, d_labels, bytes, cudaMemcpyDeviceToDevice, m->stream));
-      if (rec.exec == nullptr && record_step(m, B, S, &rec) != QZO_OK) m->use_graphs = false;
+      if (rec.exec == nullptr && record_forwards(m, B, S, &rec) != QZO_OK) m->use_graphs = false;
       if (rec.exec != nullptr) {
-        QZO_TRY(launch_set_step_params(m->sp_dev, seed, eps, lr, 0.0f, clip, m->stream));
+        QZO_TRY(launch_set_step_params(m->sp_dev, seed, eps, m->stream));
         QZO_CUDA_TRY(cudaGraphLaunch(rec.exec, m->stream));
         add_launches(rec.launches);
         m->last_T = rec.rows;
-        return h_out ? read_step_result(m, h_out) : QZO_OK;
+        if (d_sums != m->sums)
+          QZO_CUDA_TRY(cudaMemcpyAsync(d_sums, m->sums, 4 * sizeof(float), cudaMemcpyDeviceToDevice, m->stream));
+        return QZO_OK;
       }
       d_tokens = m->tok_dev;
       d_labels = m->lab_dev;
     }
     rec.seen = true;                          // the first step of a shape runs the direct way
   }
-  QZO_TRY(step_begin(m, d_tokens, d_labels, B, S, seed, eps, m->sums));
+  return step_begin(m, d_tokens, d_labels, B, S, seed, eps, d_sums);
+}
+
+int step_device(qzo_model* m, const int32_t* d_tokens, const int32_t* d_labels, int B, int S, uint64_t seed, float eps,
+                float lr, float clip, float* h_out) {
+  QZO_TRY(step_begin_replayed(m, d_tokens, d_labels, B, S, seed, eps, m->sums));
   return step_finish(m, m->sums, seed, eps, lr, clip, h_out);
 }
 
@@ -837,7 +845,7 @@ int qzo_step_begin(qzo_model* m, const int32_t* d_tokens, const int32_t* d_label
                    float eps, float* d_sums) {
   QZO_TRY(check_batch(m, d_tokens, d_labels, B, S));
   if (!(eps > 0.0f) || !d_sums || ((uintptr_t)d_sums & 15)) return QZO_ERR_BAD_ARG;
-  return step_begin(m, d_tokens, d_labels, B, S, seed, eps, d_sums);
+  return step_begin_replayed(m, d_tokens, d_labels, B, S, seed, eps, d_sums);
 }
 
 int qzo_step_finish(qzo_model* m, const float* d_sums, uint64_t seed, float eps, float lr, float clip, float* h_out) {

@@ -148,9 +148,7 @@ __global__ void unpack_kernel_layout_kernel(const uint32_t* __restrict__ wq, int
 // One thread per counter block = four consecutive scales.
 // ---------------------------------------------------------------------------------------
 __global__ void update_scales_kernel(__nv_bfloat16* __restrict__ s, int64_t count, uint64_t seed,
-                                     uint64_t index_base, float coef_host, const float* __restrict__ coef_dev,
-                                     const StepParams* __restrict__ sp) {
-  if (sp) seed = sp->seed;               // a recorded step: the seed lives on the device
+                                     uint64_t index_base, float coef_host, const float* __restrict__ coef_dev) {
   const float coef = coef_dev ? *coef_dev : coef_host;
   if (coef == 0.0f) return;            // d' = 0 (or a rejected step): scales stay bit-identical
   const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -337,11 +335,11 @@ int launch_unpack_kernel_layout(const void* d_wq, int K, int N, int8_t* d_q, cud
 }
 
 int launch_update_scales(__nv_bfloat16* d_s, int64_t count, uint64_t seed, uint64_t index_base,
-                         float coef_host, const float* coef_dev, cudaStream_t st, const StepParams* sp) {
+                         float coef_host, const float* coef_dev, cudaStream_t st) {
   if (count == 0) return QZO_OK;
   const int64_t threads_total = ceil_div64(count, 4);
   QZO_LAUNCH(update_scales_kernel, dim3((unsigned)ceil_div64(threads_total, 256)), dim3(256), 0, st,
-             d_s, count, seed, index_base, coef_host, coef_dev, sp);
+             d_s, count, seed, index_base, coef_host, coef_dev);
   return QZO_OK;
 }
 

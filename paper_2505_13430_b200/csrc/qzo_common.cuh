@@ -33,11 +33,11 @@ void set_last_cuda_error(cudaError_t e);
 constexpr int kStatusTimeout = 1;    // a bounded device-side wait expired in some launch
 constexpr int kStatusBadToken = 2;   // a token id outside [0, vocab) reached the embedding
 
-// Per-step quantities of a recorded step (a CUDA graph that is replayed): its kernels read them from
-// device memory, so that one recorded launch sequence serves every seed and every step size.
+// Per-step quantities of a recorded forward (a CUDA graph that is replayed): the GEMM kernels read them
+// from device memory, so that one recorded launch sequence serves every seed and every eps.
 struct StepParams {
   unsigned long long seed;
-  float eps, lr, lr_dense, clip;
+  float eps;
 };
 
 constexpr int kGroup = 128;          // rows of one quantisation group (paper: group 128)

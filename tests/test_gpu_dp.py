@@ -27,9 +27,14 @@ def test_single_rank_dp_step_equals_qzo_step():
     ref = gm.qzo_step(tok_d, lab_d, 42, c["eps"], c["lr"] * 50, c["clip"])
     after_ref = gm.scales.clone()
     gm.scales.copy_(before)
-    got = dp.dp_step(gm, tok_d, lab_d, 42, c["eps"], c["lr"] * 50, c["clip"])
-    assert got == ref
-    assert torch.equal(gm.scales.view(torch.int16), after_ref.view(torch.int16))
+    # three times: the first data-parallel step of the shape replays what qzo_step left recorded or records
+    # itself; every one of them must reproduce the direct step
+    for _ in range(3):
+        gm.scales.copy_(before)
+        got = dp.dp_step(gm, tok_d, lab_d, 42, c["eps"], c["lr"] * 50, c["clip"])
+        assert got == ref
+        assert torch.equal(gm.scales.view(torch.int16), after_ref.view(torch.int16))
+    assert gm.qzo_recorded_step_count() == 1
     assert not torch.equal(after_ref.view(torch.int16), before.view(torch.int16))
     gm.close()
 
