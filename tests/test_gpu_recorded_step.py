@@ -1,5 +1,5 @@
-"""qzo_step replayed from a recorded launch sequence (a CUDA graph per batch shape, its kernels reading seed,
-eps, lr and clip from device memory) against the same steps issued launch by launch: losses, d, d' and the
+"""qzo_step with its two forwards replayed from a recorded launch sequence (a CUDA graph per batch shape, its
+GEMMs reading seed and eps from device memory) against the same steps issued launch by launch: losses, d, d' and the
 scales must agree bit for bit, step after step, across seeds, step sizes and batch shapes."""
 import pytest
 import torch
