@@ -126,6 +126,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// One test of the barrier that never suspends the thread (try_wait may park it for a while when the phase
+// is not complete): for a warp whose lanes look at several barriers, most of them not due yet.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 // Up to 1024 polls of the barrier in a short loop; true when the phase completed.
 __device__ __forceinline__ bool mbar_poll(uint32_t bar, uint32_t parity) {
   uint32_t done;
@@ -350,7 +363,10 @@ struct SmemPlan {
   // bytes of one slot of the ring that the A producer fills: int4 path: nibbles and scales of a group (the
   // de-quantised operand lives in tensor memory); bf16 path: the 16 KiB tile the MMA reads
   static constexpr int kNibBytes = DEQUANT ? kNibSlotBytes : kAStageBytes;
-  static constexpr int kBStages = DEQUANT ? cmin(8, (kSmemBudget - kFixedBytes - kASlots * kNibBytes) / kXTileBytes) / kBGroup * kBGroup : 4;
+  // up to 8 stages; 16 where a stage is at most 4 KiB (token tiles up to 32): there a slot's round trip (its
+  // group's MMAs retire, the producer sees it, the tile arrives from L2) is longer than four groups last
+  static constexpr int kBStagesMax = (DEQUANT && TOK <= 32) ? 16 : 8;
+  static constexpr int kBStages = DEQUANT ? cmin(kBStagesMax, (kSmemBudget - kFixedBytes - kASlots * kNibBytes) / kXTileBytes) / kBGroup * kBGroup : 4;
   static constexpr int kBSlots = kBStages / kBGroup;
   static_assert(kBSlots >= 2 && kASlots >= 2, "pipelines need at least two stages");
   // int4 path: the nibble ring is deeper than the tensor-memory stages wherever shared memory is left (small
@@ -430,6 +446,10 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
   constexpr int kBStages = Plan::kBStages;
   constexpr int kBSlots = Plan::kBSlots;
   constexpr int kBGroup = Plan::kBGroup;
+  // Token tiles up to 128: a slot of either ring is one quantisation group, and both are free when the group's
+  // MMAs have retired, so the issuer signs ONE barrier per group (a tcgen05.commit costs the issuing thread
+  // about as much as four MMAs): the tensor-memory slot's "empty" barrier, which the B producer watches too.
+  constexpr bool kMergedRelease = DEQUANT && kAGroup == 2 && kBGroup == 2;
   constexpr uint32_t kAccCols = Plan::kAccCols;
   constexpr uint32_t kTmemCols = Plan::kTmemCols;
   extern __shared__ uint8_t smem_raw[];
@@ -524,7 +544,18 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         if (is_b) {
           for (int it = 0; it < w.nkb; it += kBGroup) {
             const int nk = min(kBGroup, w.nkb - it);          // k-blocks of this slot
-            if (!mbar_wait(bar_b_empty(ring.s), ring.ph ^ 1u, abort_flag, wait_limit)) { ok = false; break; }
+            if (kMergedRelease) {
+              // the slot's previous group (kBSlots groups back) is released by that group's tensor-memory
+              // slot: one commit of the issuer frees both
+              const int x = issued - kBSlots;
+              if (x >= 0 && !mbar_wait(bar_a_empty(x % kASlots), (uint32_t)(x / kASlots) & 1u, abort_flag, wait_limit)) {
+                ok = false;
+                break;
+              }
+            } else if (!mbar_wait(bar_b_empty(ring.s), ring.ph ^ 1u, abort_flag, wait_limit)) {
+              ok = false;
+              break;
+            }
             mbar_arrive_expect_tx(bar_b_full(ring.s), (uint32_t)(nk * Plan::kXTileBytes));
             for (int j = 0; j < nk; ++j)
               tma_load_2d(base + Plan::kOffB + (ring.s * kBGroup + j) * Plan::kXTileBytes, &tmap_x, bar_b_full(ring.s),
@@ -592,14 +623,50 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     const uint64_t bdesc0 = umma_desc_k_major_sw128(base + Plan::kOffB);   // stage s: start address + s * tile bytes
     Ring ra, rb;
     int itg = 0;
-    for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x) {
+    int seen = 0;                                             // k-blocks the watch warp had published at the last look
+    // Token tiles up to 128: one pass of the loop per quantisation group (its two k-blocks sit side by side in both
+    // rings): eight MMAs and one commit with as little around them as possible.  This thread's instruction stream
+    // is what the small-token GEMM waits for (it shares its scheduler with the de-quantisers).
+    for (int u = blockIdx.x; kMergedRelease && u < p.total_units && ok; u += gridDim.x) {
+      const Unit w = decode_unit(p, u, TOK);
+      const int ngroups = (w.nkb + 1) >> 1;
+      for (int g = 0; g < ngroups; ++g) {
+        const int nk = (2 * g + 1 < w.nkb) ? 2 : 1;
+        if (seen < itg + nk) {
+          seen = ld_acquire_shared(ready_addr);
+          if (seen >= 0 && seen < itg + nk) {
+            const long long t0 = clock64();
+            do {
+              seen = ld_acquire_shared(ready_addr);
+            } while (seen >= 0 && seen < itg + nk && clock64() - t0 < wait_limit);
+          }
+          if (seen < itg + nk) { ok = false; break; }         // the watch warp gave up (-1), or the limit expired
+          tcgen05_fence_after();
+        }
+        if (leader) {
+          const uint32_t a_tmem = tmem_d + kAccCols + (uint32_t)(ra.s * kAGroup * kATmemColsPerStage);
+          const uint64_t bdesc = bdesc0 + (uint64_t)(rb.s * kBGroup * (Plan::kXTileBytes >> 4));
+          umma_bf16_tmem_a_x4(tmem_d, a_tmem, bdesc, idesc, g > 0 ? 1u : 0u);
+          if (nk == 2) umma_bf16_tmem_a_x4(tmem_d, a_tmem + kATmemColsPerStage, bdesc + (uint64_t)(Plan::kXTileBytes >> 4), idesc, 1u);
+          umma_commit(bar_a_empty(ra.s));                     // frees the group's slot in both rings
+        }
+        itg += nk;
+        ra.next(kASlots);
+        rb.next(kBSlots);
+      }
+      if (!ok) break;
+      if (leader) umma_commit(bar_acc_full);
+      __syncwarp();
+    }
+    for (int u = blockIdx.x; !kMergedRelease && u < p.total_units && ok; u += gridDim.x) {
       const Unit w = decode_unit(p, u, TOK);
       for (int it = 0; it < w.nkb; ++it, ++itg) {
         const int j = it % kAGroup;                           // position inside the A slot
-        {
+        if (seen <= itg) {
           // wait (bounded) until the watch warp has seen this k-block's operands ready and, for the
-          // first k-block of a unit, the accumulator drained
-          int seen = ld_acquire_shared(ready_addr);
+          // first k-block of a unit, the accumulator drained.  The count it publishes often covers several
+          // k-blocks: the issuer asks again only when it has used up what it last saw.
+          seen = ld_acquire_shared(ready_addr);
           if (seen >= 0 && seen <= itg) {
             const long long t0 = clock64();
             do {
@@ -607,8 +674,8 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             } while (seen >= 0 && seen <= itg && clock64() - t0 < wait_limit);
           }
           if (seen <= itg) { ok = false; break; }             // the watch warp gave up (-1), or the limit expired
+          tcgen05_fence_after();
         }
-        tcgen05_fence_after();
         const bool slot_done = j == kAGroup - 1 || it == w.nkb - 1;
         const int jb = it % kBGroup;                          // position inside the B slot
         const bool bslot_done = jb == kBGroup - 1 || it == w.nkb - 1;
@@ -625,7 +692,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
               umma_bf16(tmem_d, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
                         (it > 0 || k > 0) ? 1u : 0u);
           }
-          if (bslot_done) umma_commit(bar_b_empty(rb.s)); // releases the B slot
+          if (bslot_done && !kMergedRelease) umma_commit(bar_b_empty(rb.s)); // releases the B slot
           if (slot_done) umma_commit(DEQUANT ? bar_a_empty(ra.s) : bar_nib_free(ra.s));  // and, after its last k-block, the A slot
         }
         if (slot_done) ra.next(kASlots);
@@ -637,11 +704,58 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     if (!ok) *abort_flag = 1;
   } else if (warp == kWatchWarp) {
     // ------------------------------------------------------------------ watch warp
-    // Performs the (bounded) mbarrier waits the MMA issuer depends on, one k-block ahead of it in
-    // time, and publishes the count of ready k-blocks.
+    // Performs the (bounded) mbarrier waits the MMA issuer depends on, ahead of it in time, and publishes
+    // the count of ready k-blocks.
     Ring ra, rb;
     int useq = 0, itg = 0;
-    for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x, ++useq) {
+    // Slots of one quantisation group in both rings (token tiles up to 128): the lanes test the barriers of
+    // the next kLook groups at once and the warp publishes every group up to the first one that is not ready,
+    // so that what this warp costs per group (a test, a ballot, a release) is paid once per batch: a warp
+    // that tests one barrier after the other needs about as long per group as the issuer does, and the two
+    // then take turns instead of overlapping.
+    constexpr bool kBatchedWatch = DEQUANT && kAGroup == 2 && kBGroup == 2;
+    constexpr int kLook = kASlots < kBSlots ? kASlots : kBSlots;
+    int gig = 0;                          // quantisation groups of this CTA's earlier units
+    for (int u = blockIdx.x; kBatchedWatch && u < p.total_units && ok; u += gridDim.x, ++useq) {
+      const Unit w = decode_unit(p, u, TOK);
+      const int ngroups = (w.nkb + 1) >> 1;
+      // the epilogue warps must have drained the previous unit's accumulator
+      bool good = mbar_wait(bar_acc_empty, ((uint32_t)useq & 1u) ^ 1u, abort_flag, wait_limit);
+      int done = 0;                       // groups of this unit published so far
+      long long t0 = 0;
+      bool timing = false;
+      while (good && done < ngroups) {
+        const int cand = done + lane;     // this lane's group of the unit
+        bool rdy = false;
+        if (lane < kLook && cand < ngroups) {
+          // group gs uses slot gs % slots in round gs / slots of either ring; the groups of earlier rounds of a
+          // slot lie before the head (kLook <= slots), so their phases are complete
+          const int gs = gig + cand;
+          rdy = mbar_test_wait(bar_a_deq(gs % kASlots), (uint32_t)(gs / kASlots) & 1u) &&
+                mbar_test_wait(bar_b_full(gs % kBSlots), (uint32_t)(gs / kBSlots) & 1u);
+        }
+        const uint32_t mask = __ballot_sync(0xffffffffu, rdy);
+        const int n = __ffs((int)~mask) - 1;            // consecutive ready groups from the head
+        if (n > 0) {
+          done += n;
+          itg += 2 * n - ((done == ngroups && (w.nkb & 1)) ? 1 : 0);   // the last group of an odd K has one k-block
+          if (lane == 0) st_release_shared(ready_addr, itg);
+          timing = false;
+        } else if (!timing) {
+          t0 = clock64();
+          timing = true;
+        } else if (*abort_flag || clock64() - t0 > wait_limit) {
+          good = false;
+        }
+      }
+      if (!good) {
+        if (lane == 0) st_release_shared(ready_addr, -1);
+        ok = false;
+        break;
+      }
+      gig += ngroups;
+    }
+    for (int u = blockIdx.x; !kBatchedWatch && u < p.total_units && ok; u += gridDim.x, ++useq) {
       const Unit w = decode_unit(p, u, TOK);
       for (int it = 0; it < w.nkb; ++it) {
         const int j = it % kAGroup;
