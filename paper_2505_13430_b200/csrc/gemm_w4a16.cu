@@ -18,9 +18,11 @@
 //
 // Warp roles (25 warps):
 //   warp 0       TMA producer of the B ring: activation tiles (2-D tensor map, 128-byte swizzle)
-//   warp 1       MMA issuer (one elected lane), owns the TMEM allocation
+//   warp 1       MMA issuer (one elected lane), owns the TMEM allocation; token tiles up to 128: eight MMAs and
+//                one commit per quantisation group (the commit frees the group's slot in both rings)
 //   warp 2       producer of the A ring: packed int4 tiles (one 8 KiB bulk copy per quantisation group)
-//   warp 3       watch warp: does the mbarrier waits the issuer depends on and publishes a count
+//   warp 3       watch warp: does the mbarrier waits the issuer depends on and publishes a count; token tiles up
+//                to 128: its lanes test the barriers of the next groups at once and it publishes in batches
 //   warps 4-7    scale warps: Philox4x32-10 + Box-Muller, s' = s + sign eps z in fp32, split
 //                into bf16 hi + lo parts, written next to the nibbles of the group's A slot
 //   warps 8-15   de-quantisers: nibbles -> bf16 (u - 8) * s' written to the A stages in TMEM; two teams
