@@ -16,7 +16,7 @@
 // the activations (q, k, v or gate, up) are served by one launch; the logical scale index of a
 // scale never depends on that grouping.
 //
-// Warp roles (25 warps):
+// Warp roles (25 warps; 29 at token tiles up to 128):
 //   warp 0       TMA producer of the B ring: activation tiles (2-D tensor map, 128-byte swizzle)
 //   warp 1       MMA issuer (one elected lane), owns the TMEM allocation; token tiles up to 128: eight MMAs and
 //                one commit per quantisation group (the commit frees the group's slot in both rings)
@@ -25,11 +25,11 @@
 //                to 128: its lanes test the barriers of the next groups at once and it publishes in batches
 //   warps 4-7    scale warps: Philox4x32-10 + Box-Muller, s' = s + sign eps z in fp32, split
 //                into bf16 hi + lo parts, written next to the nibbles of the group's A slot
-//   warps 8-15   de-quantisers: nibbles -> bf16 (u - 8) * s' written to the A stages in TMEM; two teams
-//                of four warps take alternate quantisation groups
-//   warps 16-23  epilogue: TMEM -> registers (+ bias) -> bf16 rows in shared memory, 32 tokens per pass
+//   warps 8-15   de-quantisers: nibbles -> bf16 (u - 8) * s' written to the A stages in TMEM; teams of four
+//    (8-19)      warps take the quantisation groups in turn: two teams at 256-token tiles, three below
+//   next 8       epilogue: TMEM -> registers (+ bias) -> bf16 rows in shared memory, 32 tokens per pass
 //                (the last passes of a full tile wait in registers: the accumulator is released first)
-//   warp 24      store warp: issues the TMA store of every staged pass (three staging buffers), so
+//   last warp    store warp: issues the TMA store of every staged pass (three staging buffers), so
 //                that the warps draining the single accumulator never wait for a store to be issued
 // Every wait on an mbarrier is bounded; when a wait expires the CTA records an error in
 // the status word, drains its copies and leaves through the common exit (TMEM is freed).
@@ -49,16 +49,24 @@ namespace {
 constexpr int kATmemColsPerStage = kBlockK / 2;   // 64 bf16 along K = 32 TMEM columns of 32 bits
 constexpr int kMaxASlots = 7;         // A-ring slots (quantisation groups in flight); each holds its perturbed scales
 constexpr int kNumScaleWarps = 4;
-constexpr int kNumDeqWarps = 8;
 constexpr int kNumEpiWarps = 8;
 constexpr int kAProducerWarp = 2;
 constexpr int kWatchWarp = 3;          // waits on the mbarriers on behalf of the MMA issuer
 constexpr int kFirstScaleWarp = 4;
 constexpr int kFirstDeqWarp = kFirstScaleWarp + kNumScaleWarps;
-constexpr int kFirstEpiWarp = kFirstDeqWarp + kNumDeqWarps;
-constexpr int kStoreWarp = kFirstEpiWarp + kNumEpiWarps;   // issues the TMA stores of the finished tiles
-constexpr int kNumWarps = kStoreWarp + 1;
-constexpr int kThreads = kNumWarps * 32;
+// De-quantiser teams of four warps (one warp per tensor-memory lane quadrant), taking quantisation groups in turn:
+// two at 256-token tiles (72 registers per thread there; a third team would not fit the register file) and
+// for bf16 weights (where they idle), three at token tiles up to 128, where every role gets an issue slot only now
+// and then and a third team shortens the de-quantisers' turn-around.  The warps after them follow.
+template <int TOK, int WMODE>
+struct Roles {
+  static constexpr int kDeqTeams = (WMODE != 0 && TOK <= 128) ? 3 : 2;
+  static constexpr int kNumDeqWarps = 4 * kDeqTeams;
+  static constexpr int kFirstEpiWarp = kFirstDeqWarp + kNumDeqWarps;
+  static constexpr int kStoreWarp = kFirstEpiWarp + kNumEpiWarps;   // issues the TMA stores of the finished tiles
+  static constexpr int kNumWarps = kStoreWarp + 1;
+  static constexpr int kThreads = kNumWarps * 32;
+};
 constexpr long long kWaitLimitCycles = 4000000000LL;   // ~2 s at boost clock
 constexpr int kSmemBudget = 227 * 1024;
 
@@ -434,11 +442,15 @@ struct Ring {
 // WMODE (WeightMode): kWInt4 / kWTable16: A operand produced from packed 4-bit codes + perturbed scales;
 // kWBf16: A operand is a bf16 [N][K] row-major matrix loaded through tmap_w (lm_head).
 template <int TOK, int WMODE, int OUT_MODE>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__((Roles<TOK, WMODE>::kThreads), 1)
 w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                   const __grid_constant__ CUtensorMap tmap_y0, const __grid_constant__ CUtensorMap tmap_y1,
                   const __grid_constant__ CUtensorMap tmap_y2, const __grid_constant__ GemmParams p) {
   using Plan = SmemPlan<TOK, WMODE, OUT_MODE>;
+  using R = Roles<TOK, WMODE>;
+  constexpr int kDeqTeams = R::kDeqTeams;
+  constexpr int kFirstEpiWarp = R::kFirstEpiWarp;
+  constexpr int kStoreWarp = R::kStoreWarp;
   constexpr bool DEQUANT = Plan::DEQUANT;
   constexpr bool LUT = Plan::LUT;
   constexpr int kScaleRows = Plan::kScaleRows;
@@ -506,10 +518,10 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
       // int4 path: the slot is full when its nibbles have landed AND its perturbed scales are written
       mbar_init(bar_nib_full(s), DEQUANT ? 2 : 1);
       mbar_init(bar_nib_raw(s), 1);
-      mbar_init(bar_nib_free(s), DEQUANT ? kNumDeqWarps / 2 : 1);   // one team of four de-quantiser warps per group
+      mbar_init(bar_nib_free(s), DEQUANT ? 4 : 1);   // one team of four de-quantiser warps per group
     }
     for (int s = 0; s < kASlots; ++s) {
-      mbar_init(bar_a_deq(s), kNumDeqWarps / 2);
+      mbar_init(bar_a_deq(s), 4);
       mbar_init(bar_a_empty(s), 1);
     }
     mbar_init(bar_acc_full, 1);
@@ -856,9 +868,9 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
   } else if (warp < kFirstEpiWarp) {
     // ------------------------------------------------------------------ de-quantisers
     if (DEQUANT) {
-      const int dt = threadIdx.x - kFirstDeqWarp * 32;      // 0..255
+      const int dt = threadIdx.x - kFirstDeqWarp * 32;      // 0 .. 128 kDeqTeams - 1
       const int r = (warp & 3) * 32 + lane;                 // row of the tile = TMEM lane this warp may access
-      const int team = dt >> 7;                             // two teams of four warps take alternate groups
+      const int team = dt >> 7;                             // the teams of four warps take the groups in turn
       const __nv_bfloat162 magic_bias = __halves2bfloat162(__float2bfloat16_rn(136.0f), __float2bfloat16_rn(136.0f));
       __nv_bfloat162 s_hi, s_lo;
       *reinterpret_cast<uint32_t*>(&s_hi) = 0u;
@@ -896,7 +908,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
       for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x) {
         const Unit w = decode_unit(p, u, TOK);
         for (int it = 0; it < w.nkb; it += 2, ++gig) {
-          if ((gig & 1) != team) continue;                    // the other team's group
+          if ((gig % kDeqTeams) != team) continue;            // another team's group
           const int nslot = gig % kNibSlots;                  // nibble-ring slot of this group
           const uint32_t nph = (uint32_t)(gig / kNibSlots) & 1u;
           const int slot = gig % kASlots;                     // tensor-memory slot = one quantisation group (two k-blocks)
@@ -1183,7 +1195,7 @@ int launch_one(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorMap* 
   if (first_use_on_device(configured))
     QZO_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Plan::kDynamicBytes));
   const int grid = p.total_units < sm_count() ? p.total_units : sm_count();
-  QZO_LAUNCH(kern, dim3(grid), dim3(kThreads), Plan::kDynamicBytes, st, tx, tw, ty[0], ty[1], ty[2], p);
+  QZO_LAUNCH(kern, dim3(grid), dim3(Roles<TOK, WMODE>::kThreads), Plan::kDynamicBytes, st, tx, tw, ty[0], ty[1], ty[2], p);
   return QZO_OK;
 }
 
