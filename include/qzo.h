@@ -122,6 +122,18 @@ int qzo_perturbed_gemm_table16(const void* d_x_bf16, const void* d_codes, const 
                                uint64_t seed, uint64_t scale_index_base, int sign, float eps,
                                void* d_workspace, size_t workspace_bytes, int* d_status, void* stream);
 
+/* The same table prologue for weights whose only continuous parameter is one scale per OUTPUT CHANNEL (the
+ * paper's codebook setting, Sec. 4.1: AQLM-style codebook weights, of which QZO tunes the channel-wise scales;
+ * here with a 16-entry scalar table standing in for the codebook):
+ *   Y[t][n] = (s[n] + sign eps z_i) sum_k X[t][k] table[c[k][n]] (+ bias[n]),  i = scale_index_base + n.
+ * d_scales bf16 [N]; everything else as qzo_perturbed_gemm_table16.  The seeded update of such scales is
+ * qzo_update_scales_flat over N entries. */
+int qzo_perturbed_gemm_codebook16_channelwise(const void* d_x_bf16, const void* d_codes, const void* d_scales_bf16,
+                                              const float* h_table16, const float* d_bias, void* d_y_bf16,
+                                              int M, int K, int N, uint64_t seed, uint64_t scale_index_base,
+                                              int sign, float eps, void* d_workspace, size_t workspace_bytes,
+                                              int* d_status, void* stream);
+
 /* The same linear for callers that must not allocate device memory and have no workspace to
  * lend: for example a serving process that gave all device memory to its own pool when it
  * started, or a latency-critical loop in which the device-wide synchronisation of an allocation

@@ -61,19 +61,26 @@ def perturbed_linear_samples(x_rows, q_cols, s_cols, cols, N, seed, index_base, 
 TABLE_BLOCK = 64
 
 
-def perturbed_linear_table16(x, codes, s, table, seed, index_base, sign, eps, bias=None):
+def perturbed_linear_table16(x, codes, s, table, seed, index_base, sign, eps, bias=None, channelwise=False):
     """Block-scaled 16-entry codebook weights (NF4-style storage): w[k][n] = s'[k // 64][n] * table[codes[k][n]],
     codes in [0, 15], one scale per block of 64 consecutive input rows of an output column, and
     s' = s + sign*eps*z with z at index index_base + b*N + n for scale [b][n] (Eq. 5 on the format's
-    continuous scales; the codes and the table stay fixed).  Y = X W (+ bias), fp64."""
+    continuous scales; the codes and the table stay fixed).  Y = X W (+ bias), fp64.
+
+    channelwise: s is [1][N], one scale per output channel (the codebook setting of Sec. 4.1, where the
+    channel-wise scales are what QZO tunes): w[k][n] = s'[n] * table[codes[k][n]], z at index_base + n."""
     x = np.asarray(x, dtype=np.float64)
     codes = np.asarray(codes)
     table = np.asarray(table, dtype=np.float64)
     assert table.shape == (16,) and codes.min() >= 0 and codes.max() <= 15
     K = codes.shape[0]
     sp = perturbed_scales(s, seed, index_base, sign, eps)
-    assert sp.shape[0] == (K + TABLE_BLOCK - 1) // TABLE_BLOCK
-    w = sp[np.arange(K) // TABLE_BLOCK] * table[codes]
+    if channelwise:
+        assert sp.shape[0] == 1
+        w = sp[np.zeros(K, dtype=np.int64)] * table[codes]
+    else:
+        assert sp.shape[0] == (K + TABLE_BLOCK - 1) // TABLE_BLOCK
+        w = sp[np.arange(K) // TABLE_BLOCK] * table[codes]
     y = x @ w
     if bias is not None:
         y = y + np.asarray(bias, dtype=np.float64)[None, :]

@@ -108,6 +108,7 @@ struct GemmParams {
   int pair_rows;                  // > 0: token rows from this one on take -sign_eps (both passes of a step in one launch)
   int* status;
   long long wait_limit;           // cycles after which a device-side wait gives up
+  int scale_row_mul;              // 1: one row of scales per group / block of k; 0: one row for all k (channel-wise scales)
   int skip_group;                 // >= 0 (tests only): the A producer announces this group's copies but does not issue them
   float lut[16];                  // table mode: the 16 codebook values (a nibble is an index into them)
 };
@@ -600,7 +601,7 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 const int row0 = LUT ? kb : (kb >> 1);
                 mbar_arrive_expect_tx(bar_nib_raw(ring.s), raw_bytes * (uint32_t)rows);
                 for (int j = 0; j < rows && !skip; ++j)
-                  bulk_load(dst + Plan::kOffRawInSlot + j * kRawScaleBytes, L.scales + (size_t)(row0 + j) * L.N + w.n0, raw_bytes,
+                  bulk_load(dst + Plan::kOffRawInSlot + j * kRawScaleBytes, L.scales + (size_t)((row0 + j) * p.scale_row_mul) * L.N + w.n0, raw_bytes,
                             bar_nib_raw(ring.s));
               }
             } else {
@@ -823,10 +824,10 @@ w4a16_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             raw[j] = make_uint2(0u, 0u);
             if (live && j < rows) {
               if (sign_eps != 0.0f) {
-                const uint64_t i0 = L.idx_base + (uint64_t)(row0 + j) * (uint64_t)L.N + (uint64_t)(w.n0 + r0);
+                const uint64_t i0 = L.idx_base + (uint64_t)((row0 + j) * p.scale_row_mul) * (uint64_t)L.N + (uint64_t)(w.n0 + r0);
                 normals_of_block(seed, i0 >> 2, z[j]);
               }
-              if (!Plan::kRawViaCopy) raw[j] = *reinterpret_cast<const uint2*>(L.scales + (size_t)(row0 + j) * L.N + w.n0 + r0);
+              if (!Plan::kRawViaCopy) raw[j] = *reinterpret_cast<const uint2*>(L.scales + (size_t)((row0 + j) * p.scale_row_mul) * L.N + w.n0 + r0);
             }
           }
           uint8_t* const slot_mem = smem + Plan::kOffA + slot * Plan::kNibBytes;
@@ -1278,9 +1279,10 @@ size_t gemm_workspace_bytes(int M, int K, int N, int pair_rows) {
 // lut16 (host, 16 floats) non-null: table mode: the nibbles index that table and the scales are [ceil(K/64)][N], one
 // row per block of 64 k; null: int4 with one row of scales per group of 128 k.
 // d_sp (device) non-null: seed and eps are read from it when the kernel runs, the arguments of those names are ignored.
+// channel_scales: the scales are one row [N] for all k (channel-wise), index idx_base + n.
 int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const GemmLinear* lins, int n_lin,
                                 uint64_t seed, int sign, float eps, int pair_rows, void* d_ws, size_t ws_bytes,
-                                int* d_status, cudaStream_t st, const float* lut16, const StepParams* d_sp) {
+                                int* d_status, cudaStream_t st, const float* lut16, const StepParams* d_sp, bool channel_scales) {
   if (M <= 0 || K <= 0 || (K % 8) != 0 || n_lin < 1 || n_lin > kMaxGroupedLinears) return QZO_ERR_BAD_ARG;
   if (pair_rows != 0 && !paired_rows_ok(M, pair_rows)) return QZO_ERR_BAD_ARG;
   for (int j = 0; j < n_lin; ++j)
@@ -1297,7 +1299,7 @@ int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const Ge
     if (any_split) {
       for (int j = 0; j < n_lin; ++j)
         QZO_TRY(launch_perturbed_gemm_group(d_x, M, K, lins + j, 1, seed, sign, eps, pair_rows, d_ws, ws_bytes, d_status,
-                                            st, lut16, d_sp));
+                                            st, lut16, d_sp, channel_scales));
       return QZO_OK;
     }
   }
@@ -1315,6 +1317,7 @@ int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const Ge
   p.status = d_status;
   p.wait_limit = g_debug_wait_limit > 0 ? g_debug_wait_limit : kWaitLimitCycles;
   p.skip_group = g_debug_skip_group;
+  p.scale_row_mul = channel_scales ? 0 : 1;
   if (lut16) memcpy(p.lut, lut16, sizeof(p.lut));
   const int splits = (n_lin == 1) ? gemm_splits_tok(m_plan, K, lins[0].N, tok) : 1;
   for (int j = 0; j < n_lin; ++j) {

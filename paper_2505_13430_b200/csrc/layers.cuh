@@ -47,11 +47,11 @@ struct GemmLinear {
 // launch serves both passes of a step; allowed when paired_rows_ok(M, pair_rows): pair_rows in {16, 32, 64, 128} or a multiple of 256.
 bool paired_rows_ok(int M, int pair_rows);
 // lut16 (host pointer to 16 floats, or null): table mode, see gemm_w4a16.cu; d_sp (device, or null): seed and eps
-// are read from it by the kernel instead of the arguments
+// are read from it by the kernel instead of the arguments; channel_scales: one row of scales [N] for all k
 int launch_perturbed_gemm_group(const __nv_bfloat16* d_x, int M, int K, const GemmLinear* lins, int n_lin,
                                 uint64_t seed, int sign, float eps, int pair_rows, void* d_ws, size_t ws_bytes,
                                 int* d_status, cudaStream_t st, const float* lut16 = nullptr,
-                                const StepParams* d_sp = nullptr);
+                                const StepParams* d_sp = nullptr, bool channel_scales = false);
 // Test hook: later perturbed-GEMM launches of the calling thread use this wait limit (cycles; 0 = the normal
 // one) and withhold the copies of quantisation group `skip_group` of every CTA (-1 = none).
 void set_gemm_wait_debug(long long limit_cycles, int skip_group);

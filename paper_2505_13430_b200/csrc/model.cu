@@ -606,6 +606,26 @@ int qzo_perturbed_gemm_table16(const void* d_x_bf16, const void* d_codes, const 
                                      workspace_bytes, d_status, (cudaStream_t)stream, h_table16);
 }
 
+int qzo_perturbed_gemm_codebook16_channelwise(const void* d_x_bf16, const void* d_codes, const void* d_scales_bf16,
+                                              const float* h_table16, const float* d_bias, void* d_y_bf16, int M, int K, int N,
+                                              uint64_t seed, uint64_t scale_index_base, int sign, float eps,
+                                              void* d_workspace, size_t workspace_bytes, int* d_status, void* stream) {
+  if (!d_x_bf16 || !d_codes || !d_scales_bf16 || !d_y_bf16 || !h_table16) return QZO_ERR_BAD_ARG;
+  if (sign < -1 || sign > 1 || !(eps > 0.0f)) return QZO_ERR_BAD_ARG;
+  for (int i = 0; i < 16; ++i)
+    if (!std::isfinite(h_table16[i])) return QZO_ERR_BAD_ARG;
+  if (((uintptr_t)d_x_bf16 & 15) || ((uintptr_t)d_codes & 15) || ((uintptr_t)d_scales_bf16 & 15) ||
+      ((uintptr_t)d_y_bf16 & 15))
+    return QZO_ERR_BAD_ARG;
+  if (d_workspace && ((uintptr_t)d_workspace & 255)) return QZO_ERR_WORKSPACE;
+  QZO_TRY(check_device());
+  if (N <= 0 || (N % 8)) return QZO_ERR_BAD_ARG;
+  const GemmLinear g{d_codes, (const __nv_bfloat16*)d_scales_bf16, d_bias, (__nv_bfloat16*)d_y_bf16, N, N,
+                     scale_index_base};
+  return launch_perturbed_gemm_group((const __nv_bfloat16*)d_x_bf16, M, K, &g, 1, seed, sign, eps, 0, d_workspace,
+                                     workspace_bytes, d_status, (cudaStream_t)stream, h_table16, nullptr, true);
+}
+
 int qzo_debug_gemm_wait_expiry(const void* d_x_bf16, const void* d_wq, const void* d_scales_bf16, void* d_y_bf16, int M,
                                int K, int N, int skip_group, int64_t wait_limit_cycles, int* d_status, void* stream) {
   if (skip_group < 0 || wait_limit_cycles <= 0 || !d_status) return QZO_ERR_BAD_ARG;

@@ -27,7 +27,7 @@ EXPORTS = (
     "qzo_scale_layout", "qzo_workspace_bytes", "qzo_init_model", "qzo_free_model", "qzo_forward_loss",
     "qzo_update_scales", "qzo_step", "qzo_step_host", "qzo_debug_set_capture", "qzo_debug_layer_output",
     "qzo_device_status", "qzo_launch_count", "qzo_profile_gemms", "qzo_profile_read",
-    "qzo_step_begin", "qzo_step_finish", "qzo_get_scales", "qzo_set_scales", "qzo_debug_set_status", "qzo_use_recorded_steps", "qzo_recorded_step_count",
+    "qzo_step_begin", "qzo_step_finish", "qzo_get_scales", "qzo_set_scales", "qzo_debug_set_status", "qzo_use_recorded_steps", "qzo_recorded_step_count", "qzo_perturbed_gemm_codebook16_channelwise",
     "qzo_joint_workspace_bytes", "qzo_enable_joint_spsa", "qzo_perturbed_gemm_table16", "qzo_debug_gemm_wait_expiry",
 )
 
@@ -75,6 +75,7 @@ def _load():
         "qzo_gemm_workspace_bytes": (ci, [ci, ci, ci, P(sz)]),
         "qzo_perturbed_gemm": (ci, [vp, vp, vp, vp, vp, ci, ci, ci, u64, u64, ci, cf, vp, sz, vp, vp]),
         "qzo_perturbed_gemm_table16": (ci, [vp, vp, vp, P(cf), vp, vp, ci, ci, ci, u64, u64, ci, cf, vp, sz, vp, vp]),
+        "qzo_perturbed_gemm_codebook16_channelwise": (ci, [vp, vp, vp, P(cf), vp, vp, ci, ci, ci, u64, u64, ci, cf, vp, sz, vp, vp]),
         "qzo_debug_gemm_wait_expiry": (ci, [vp, vp, vp, vp, ci, ci, ci, ci, i64, vp, vp]),
         "qzo_perturbed_gemm_noalloc": (ci, [vp, vp, vp, vp, vp, ci, ci, ci, u64, u64, ci, cf, vp, vp]),
         "qzo_update_scales_flat": (ci, [vp, i64, u64, u64, cf, cf, cf, vp]),
@@ -226,6 +227,26 @@ def qzo_perturbed_gemm_table16(x, codes_wq, scales, table16, M, K, N, seed, scal
     _check(_lib.qzo_perturbed_gemm_table16(_ptr(x), _ptr(codes_wq), _ptr(scales), table, _ptr(bias), _ptr(y), M, K, N, seed,
                                            scale_index_base, sign, eps, _ptr(workspace), ws_bytes, _ptr(status), _stream()),
            "qzo_perturbed_gemm_table16")
+    return y
+
+
+def qzo_perturbed_gemm_codebook16_channelwise(x, codes_wq, scales, table16, M, K, N, seed, scale_index_base, sign, eps,
+                                              bias=None, y=None, workspace=None, status=None):
+    """Y = X W' for 4-bit codes into a 16-entry table with ONE bf16 scale per output channel (scales: [N]);
+    codes_wq as for qzo_perturbed_gemm_table16."""
+    _cuda(x, torch.bfloat16), _cuda(codes_wq, torch.uint8), _cuda(scales, torch.bfloat16)
+    assert scales.numel() == N
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.bfloat16, device=x.device)
+    need = qzo_gemm_workspace_bytes(M, K, N)
+    if workspace is None and need:
+        workspace = torch.empty((need,), dtype=torch.uint8, device=x.device)
+    ws_bytes = workspace.numel() if workspace is not None else 0
+    table = (ctypes.c_float * 16)(*[float(v) for v in table16])
+    _check(_lib.qzo_perturbed_gemm_codebook16_channelwise(_ptr(x), _ptr(codes_wq), _ptr(scales), table, _ptr(bias), _ptr(y),
+                                                          M, K, N, seed, scale_index_base, sign, eps, _ptr(workspace),
+                                                          ws_bytes, _ptr(status), _stream()),
+           "qzo_perturbed_gemm_codebook16_channelwise")
     return y
 
 

@@ -54,3 +54,31 @@ def test_table16_scales_take_the_seeded_update():
     ref = oqzo.update_scales_flat(s.float().numpy().reshape(-1), 11, 64, 1e-3, oqzo.ddc_clip(250.0, 100.0))
     got = dev.float().cpu().numpy()
     assert np.abs(got - ref).max() <= 2.0 ** -7 * np.abs(ref).max() and not np.array_equal(got, s.float().numpy().reshape(-1))
+
+
+@pytest.mark.parametrize("M,K,N", [(16, 256, 128), (40, 688, 688), (300, 1024, 384), (128, 4096, 512), (257, 2048, 1024)])
+def test_channelwise_codebook_gemm_matches_oracle(M, K, N):
+    # one scale per output channel (the codebook setting of Sec. 4.1): same codes, same table, scales [N]
+    from paper_2505_13430_b200 import qzo as lib
+    x, codes, s, table = inputs.table16_case(M, K, N, seed=M + K + N + 1)
+    s1 = s[:1].contiguous()
+    words = torch.from_numpy(int4.pack_int4(codes.numpy().astype(np.int64) - 8).view(np.int32)).cuda()
+    wq = lib.qzo_repack_int4(words, K, N)
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    seed, base, eps = 31 + M, 8 * (N % 5), 2e-3
+    outs = {}
+    for sign in (+1, -1, 0):
+        y = lib.qzo_perturbed_gemm_codebook16_channelwise(x.cuda(), wq, s1.cuda().reshape(-1), table.tolist(), M, K, N, seed, base,
+                                                          sign, eps, status=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        ref = olinear.perturbed_linear_table16(x.float().numpy(), codes.numpy(), s1.float().numpy(), table.numpy(),
+                                               seed, base, sign, eps, channelwise=True)
+        assert _relerr(y, ref) <= 2e-2, (M, K, N, sign, _relerr(y, ref))
+        outs[sign] = (y.float().cpu().numpy().astype(np.float64), ref)
+    d_got, d_ref = outs[+1][0] - outs[-1][0], outs[+1][1] - outs[-1][1]
+    assert np.abs(d_got - d_ref).max() <= 3e-2 * np.abs(d_ref).max() + 2.0 ** -7 * np.abs(outs[+1][1]).max()
+    # it is NOT the block-scaled call on the same memory: there the rows below the first would be read as scales
+    if K > 64:
+        blk = lib.qzo_perturbed_gemm_table16(x.cuda(), wq, s.cuda(), table.tolist(), M, K, N, seed, base, +1, eps, status=status)
+        assert not torch.equal(blk.view(torch.int16), torch.from_numpy(outs[+1][0]).bfloat16().cuda().view(torch.int16))

@@ -109,3 +109,31 @@ def test_table16_linear_brute_force_and_special_cases():
     a = linear.perturbed_linear(xx, q, s128, 1, 0, 0, 1e-3)
     b = linear.perturbed_linear_table16(xx, q + 8, np.repeat(s128, 2, axis=0), np.arange(16) - 8.0, 1, 0, 0, 1e-3)
     assert np.abs(a - b).max() <= 1e-13 * np.abs(a).max()
+
+
+def test_channelwise_codebook_linear_factors_out_of_the_contraction():
+    # One scale per output channel (the codebook setting of Sec. 4.1): the perturbed scale multiplies the whole
+    # column, so Y = (X table[codes]) * s' column by column -- a closed form the routine must reproduce --,
+    # z is indexed by the channel alone, and at sign 0 it is the block-scaled routine with equal scales in
+    # every block.
+    from paper_2505_13430_b200 import inputs
+    x, codes, s, table = inputs.table16_case(3, 200, 16, seed=4)
+    x, codes, table = x.float().numpy().astype(np.float64), codes.numpy(), table.numpy().astype(np.float64)
+    s1 = s.float().numpy()[:1]                                   # [1][N]
+    seed, base, eps = 9, 24, 3e-3
+    z = philox.normal_range(seed, base, 16).astype(np.float64)
+    plain = x @ table[codes]                                     # the contraction without any scale
+    for sign in (+1, -1, 0):
+        got = linear.perturbed_linear_table16(x, codes, s1, table, seed, base, sign, eps, channelwise=True)
+        want = plain * (s1[0].astype(np.float64) + sign * eps * z)[None, :]
+        assert np.abs(got - want).max() <= 1e-12 * np.abs(want).max()
+        brute = sum(float(x[1, k]) * (float(s1[0, 5]) + sign * eps * z[5]) * float(table[codes[k, 5]]) for k in range(200))
+        assert abs(got[1, 5] - brute) <= 1e-12 * abs(brute)
+    blocks = np.repeat(s1, 4, axis=0)                            # ceil(200 / 64) = 4 equal rows
+    a = linear.perturbed_linear_table16(x, codes, s1, table, seed, base, 0, eps, channelwise=True)
+    b = linear.perturbed_linear_table16(x, codes, blocks, table, seed, base, 0, eps)
+    assert np.abs(a - b).max() <= 1e-13 * np.abs(a).max()
+    # a different channel's z must not leak in: shifting the base by one channel shifts which z a column gets
+    c = linear.perturbed_linear_table16(x, codes, s1, table, seed, base + 4, +1, eps, channelwise=True)
+    z4 = philox.normal_range(seed, base + 4, 16).astype(np.float64)
+    assert np.abs(c - plain * (s1[0] + eps * z4)[None, :]).max() <= 1e-12 * np.abs(c).max()
