@@ -62,3 +62,41 @@ def test_two_replicas_with_added_loss_sums_follow_the_whole_batch_step():
         assert torch.equal(ranks[0].scales.view(torch.int16), whole.scales.view(torch.int16))
     for m in ranks + [whole]:
         m.close()
+
+
+def test_seed_per_rank_step_matches_the_oracle_and_keeps_replicas_identical():
+    # Two "ranks" emulated one after the other on one GPU (nothing waits on anything): rank r perturbs with
+    # seed base + r on its half of the batch; both then apply rank 0's update and rank 1's update in that order,
+    # each from that rank's own loss sums.  Both replicas must end bit-identical, the losses must be the
+    # oracle's for (half, seed), and the scales must be the oracle's after the same two updates.
+    import numpy as np
+    from oracle import model as omodel, qzo as oqzo
+    from tests.helpers import build_oracle_model, loss_tolerance
+    qzo, cfg, c, raw, tok, lab = _tiny()
+    om = build_oracle_model(raw)
+    T = c["batch"] * c["seq"]
+    ranks = [qzo.build_model_from_raw(raw, T) for _ in range(2)]
+    base, eps, lr_each, clip = 300, c["eps"], c["lr"] * 25, c["clip"]
+    half = c["batch"] // 2
+    halves = [(tok[r * half:(r + 1) * half].contiguous(), lab[r * half:(r + 1) * half].contiguous()) for r in range(2)]
+    sums = [ranks[r].qzo_step_begin(halves[r][0].cuda(), halves[r][1].cuda(), base + r, eps).clone() for r in range(2)]
+    outs = [[ranks[k].qzo_step_finish(sums[r], base + r, eps, lr_each, clip) for r in range(2)] for k in range(2)]
+    assert outs[0] == outs[1]
+    assert torch.equal(ranks[0].scales.view(torch.int16), ranks[1].scales.view(torch.int16))
+    order = omodel.LINEAR_ORDER[cfg["arch"]]
+    for r in range(2):
+        t, l = halves[r][0].numpy(), halves[r][1].numpy()
+        tol = loss_tolerance(int((l >= 0).sum()))
+        assert abs(outs[0][r][0] - omodel.forward_loss(om, t, l, base + r, +1, eps)) <= tol
+        assert abs(outs[0][r][1] - omodel.forward_loss(om, t, l, base + r, -1, eps)) <= tol
+    for r in range(2):                                       # the oracle's updates with the device's own d'
+        oqzo.update_model_scales(om, base + r, lr_each, outs[0][r][3])
+    for li in range(cfg["n_layers"]):
+        for i, nm in enumerate(order):
+            got = ranks[0].scales_of(li, i).float().cpu().numpy()
+            ref = om["layers"][li]["lin"][nm]["s"].astype(np.float32)
+            # two updates, each rounded to bf16: within one ulp each
+            assert np.all(np.abs(got - ref) <= 2.0 ** -6 * np.abs(ref) + 1e-12)
+    assert outs[0][0][3] != 0.0 or outs[0][1][3] != 0.0
+    for m in ranks:
+        m.close()
